@@ -1,0 +1,217 @@
+/*
+ * uncomp.h -- C ABI of the prefill-end KV-cache compression pass of UNComp (arXiv 2410.03090),
+ * implemented as hand-written CUDA for NVIDIA B200 (sm_100a).
+ *
+ * One pass, four calls, all asynchronous on the caller's stream and with no host synchronisation in
+ * between (budgets and offsets stay on the device):
+ *
+ *   uncomp_entropy         truncated matrix entropy / effective rank of every (batch, layer, KV head)
+ *                          key matrix                                     (paper Section 3.1 - 3.2)
+ *   uncomp_assign_budgets  per-head token budgets from the effective ranks, and the layer-group
+ *                          partition                                      (paper Section 3.3.2, 3.3.3)
+ *   uncomp_score_select    observation-window attention scores of the prefix tokens and the top
+ *                          tokens of every head within its budget         (Section 3.3.3, "Dynamic KV
+ *                                                                          Cache Eviction")
+ *   uncomp_compact         gather of the kept K / V rows into a ragged per-head cache
+ *                                                                         (Section 3.3.3; Algorithm 2,
+ *                                                                          prefill loop over heads)
+ *
+ * Conventions
+ *   - "unit" = one (batch b, layer l, KV head h); units are numbered row-major over [B, L, H].
+ *   - Pointers whose name starts with d_ are DEVICE pointers; everything else is host memory.
+ *   - The library never allocates or frees device memory.  Inputs, outputs and the workspace belong to
+ *     the caller and must stay valid until the stream work of the call has finished.
+ *   - Every call returns an int: UNCOMP_OK or a negative UNCOMP_E_* code for a synchronous, host-side
+ *     rejection (nothing was launched).  Conditions found on the device are OR-ed into a status word
+ *     that uncomp_status() reads; kernels never trap, assert or spin without a limit.
+ *   - A context is bound to one shape and one workspace and is not thread-safe; use one per stream.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ */
+#ifndef UNCOMP_H_
+#define UNCOMP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct uncomp_ctx uncomp_ctx; /* opaque */
+
+typedef enum { UNCOMP_BF16 = 0, UNCOMP_FP32 = 1 } uncomp_dtype;
+
+/* Shape of one pass.  B sequences, L layers, H KV heads, Hq query heads (a multiple of H; G = Hq / H
+ * query heads share one KV head), N tokens, head dimension d (must be 128), observation window w
+ * (1 <= w <= 64, w < N, G * w <= 512), storage type of K, V and the window queries. */
+typedef struct {
+    int32_t B, L, H, Hq, N, d, w;
+    int32_t dtype; /* uncomp_dtype */
+} uncomp_shape;
+
+/* Element strides of a [B, L, H, N, d] tensor; the d stride is 1.  Every row must start on a 16-byte
+ * boundary (base pointer 16-byte aligned, strides multiples of 16 bytes). */
+typedef struct {
+    int64_t sB, sL, sH, sN;
+} uncomp_strides;
+
+enum {
+    UNCOMP_OK = 0,
+    UNCOMP_E_NULL = -1,        /* a required pointer is NULL */
+    UNCOMP_E_SHAPE = -2,       /* unsupported shape (d != 128, N <= w, Hq % H != 0, ...) */
+    UNCOMP_E_ALIGN = -3,       /* pointer or stride not 16-byte aligned */
+    UNCOMP_E_WORKSPACE = -4,   /* workspace smaller than uncomp_workspace_bytes() */
+    UNCOMP_E_PARAM = -5,       /* invalid hyper-parameter */
+    UNCOMP_E_CUDA = -6,        /* a CUDA runtime / driver call failed; see uncomp_last_cuda_error() */
+    UNCOMP_E_LIMIT = -7        /* size beyond a documented maximum */
+};
+
+/* Bits of the device status word. */
+enum {
+    UNCOMP_STATUS_NOT_CONVERGED = 1u, /* eigenvalue multi-section hit max_iters before its tolerance */
+    UNCOMP_STATUS_TIMEOUT = 2u,       /* a bounded device-side wait expired */
+    UNCOMP_STATUS_BOUNDS = 4u         /* an index or budget check failed; the value was clamped / skipped */
+};
+
+/* Bytes of device workspace a context of this shape needs.  Pure host function.  0 on a bad shape. */
+size_t uncomp_workspace_bytes(const uncomp_shape *shape);
+
+/* Create a context over caller-owned device workspace (256-byte aligned, at least
+ * uncomp_workspace_bytes(shape) bytes).  Clears the status word with a cudaMemset and waits for it.
+ * The device current at creation must be current for every later call. */
+int uncomp_create(uncomp_ctx **out, const uncomp_shape *shape, void *d_workspace, size_t workspace_bytes);
+void uncomp_destroy(uncomp_ctx *ctx);
+
+/* ---------------------------------------------------------------------------------------------------
+ * uncomp_entropy -- Section 3.1 Eq. 1 (covariance), Lemma 2 (eigenvalue form of the matrix entropy),
+ * Section 3.2 (truncated matrix entropy H_k and truncated effective rank erank_k = exp H_k).
+ *
+ * For every unit, with X = K[b, l, h] of shape [N, d]:
+ *   C = sum_i (x_i - mean)(x_i - mean)^T            (center = 1; C = X^T X for center = 0; the factor
+ *                                                    1/(N-1) of Eq. 1 cancels below)
+ *   lambda_1 >= ... >= lambda_d  eigenvalues of C, negatives counted as 0
+ *   p_i = lambda_i / sum_{j<=k} lambda_j  (norm = 0)   or   lambda_i / trace(C)  (norm = 1)
+ *   H_k = - sum_{i<=k} p_i ln p_i ,  erank_k = exp(H_k),   k = min(k_trunc, d)
+ *
+ * bf16 input: Gram matrix on the tensor cores with fp32 accumulation; fp32 input: fp64 accumulation.
+ * The eigenvalues are computed in fp64 (Householder tridiagonalisation in shared memory, Sturm-count
+ * multi-section for the k largest).  max_iters bounds the multi-section rounds (0 = default 14); a
+ * unit that has not reached 1e-13 of its spectral radius by then sets UNCOMP_STATUS_NOT_CONVERGED
+ * and still writes its current estimate.
+ *
+ * d_K        in   [B, L, H, N, d] with strides sK, storage dtype of the shape
+ * d_entropy  out  [B, L, H] float, H_k
+ * d_erank    out  [B, L, H] float, erank_k; may be NULL
+ * d_spectrum out  [B, L, H, k] double, the k largest eigenvalues of C (unnormalised); may be NULL
+ * ------------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t k_trunc;   /* >= 1 */
+    int32_t center;    /* 1 = Eq. 1 (centred), 0 = uncentred */
+    int32_t norm;      /* 0 = normalise over the k kept eigenvalues, 1 = over the whole trace */
+    int32_t max_iters; /* multi-section rounds, 0 = default */
+} uncomp_entropy_params;
+
+int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const uncomp_entropy_params *params,
+                   float *d_entropy, float *d_erank, double *d_spectrum, void *stream);
+
+/* ---------------------------------------------------------------------------------------------------
+ * uncomp_assign_budgets -- Section 3.3.3 "Head-Group Compression": heads ranked by truncated effective
+ * rank, split into M groups, group budgets N_{i,g+1} = N_{i,g} - step from n_max downwards; and
+ * Section 3.3.2 "Layer-Group Compression": Delta c_i, the stage count C and N_{i+1} = N_i + dn.
+ *
+ * Ranking set: the H heads of a layer (scope = 0) or all L*H heads of a sequence (scope = 1); n = its
+ * size.  Larger erank ranks first, ties go to the lower (layer, head) index.  Ranks
+ * [floor(g n/M), floor((g+1) n/M)) form group g.  Group target t_g = n_max - g * step with
+ * step = n (n_max - avg_budget) / sum_g(n_g g), so that the set's budgets sum to n * avg_budget
+ * exactly: heads get floor(t_g) and the remaining tokens go one each to the largest fractional parts
+ * (ties: better rank first).  All of it in exact integer arithmetic.  The window is part of a budget.
+ * d_offsets is the exclusive prefix sum of the budgets over units; d_offsets[units] = units * avg_budget.
+ *
+ * Layer partition (dn > 0): e_l = mean erank of layer l; a boundary follows layer l iff
+ * e_l - e_{l+1} > eps; d_layer_group[l] = boundaries before l; d_layer_ctx = N for group 0, else
+ * min(N, n_last + (boundaries_total - group) * dn).  dn = 0: group 0 and N everywhere.
+ *
+ * Rejected with UNCOMP_E_PARAM: M < 1, M > n, avg_budget < w, n_max < avg_budget, n_max > N, smallest
+ * group target below w.
+ *
+ * d_erank        in   [B, L, H] float
+ * d_budgets      out  [B, L, H] int32
+ * d_offsets      out  [B*L*H + 1] int64
+ * d_layer_group  out  [B, L] int32, may be NULL
+ * d_layer_ctx    out  [B, L] int32, may be NULL
+ * ------------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t avg_budget; /* average tokens kept per head, window included */
+    int32_t M;          /* head groups */
+    int32_t n_max;      /* budget of the group with the largest erank (paper: N_{i,1}) */
+    int32_t scope;      /* 0 = rank within each layer, 1 = rank over all heads of a sequence */
+    float eps;          /* layer partition threshold (paper: epsilon) */
+    int32_t dn;         /* context step between layer groups (paper: Delta n); 0 disables */
+    int32_t n_last;     /* context of the last layer group */
+} uncomp_budget_params;
+
+int uncomp_assign_budgets(uncomp_ctx *ctx, const float *d_erank, const uncomp_budget_params *params,
+                          int32_t *d_budgets, int64_t *d_offsets, int32_t *d_layer_group,
+                          int32_t *d_layer_ctx, void *stream);
+
+/* ---------------------------------------------------------------------------------------------------
+ * uncomp_score_select -- Section 3.3.3 "Dynamic KV Cache Eviction": the attention of the last w query
+ * positions is summed per key position and the highest-scored tokens are kept within the head's budget.
+ *
+ * For every unit and every prefix position j < N - w:
+ *   raw[j] = sum over the G query heads q of the unit and window rows i < w of softmax_j'(s_{q,i})[j],
+ *   s_{q,i}[j'] = scale * <Qw[b,l,q,i,:], K[b,l,h,j',:]>  over the causally visible j' <= N - w + i.
+ *   score[j] = max (pool_mode 0) or mean (pool_mode 1) of raw over [j - pool_kernel/2, j + pool_kernel/2]
+ *              clipped to the prefix.
+ * The budget[u] - w prefix positions with the largest score (ties: lower position) are written in
+ * ascending order to d_indices[offsets[u] ...], followed by the window positions N-w .. N-1.
+ * A budget outside [w, N] is clamped and sets UNCOMP_STATUS_BOUNDS.
+ *
+ * d_Qw       in   [B, L, Hq, w, d] contiguous, storage dtype; query head q belongs to KV head q / G
+ * d_K        in   as in uncomp_entropy
+ * d_budgets  in   [B, L, H] int32, each in [w, N]
+ * d_offsets  in   [B*L*H + 1] int64
+ * d_scores   out  [B, L, H, N - w] float, the pooled scores; may be NULL (workspace is used then)
+ * d_indices  out  [offsets[units]] int32
+ * ------------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t pool_kernel; /* odd, 1 = no pooling, at most 63 */
+    int32_t pool_mode;   /* 0 = max, 1 = mean */
+    float scale;         /* 0 means 1 / sqrt(d) */
+} uncomp_score_params;
+
+int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, uncomp_strides sK,
+                        const int32_t *d_budgets, const int64_t *d_offsets, const uncomp_score_params *params,
+                        float *d_scores, int32_t *d_indices, void *stream);
+
+/* ---------------------------------------------------------------------------------------------------
+ * uncomp_compact -- the per-head ragged cache of Section 3.3.3 ("each head maintains its context
+ * window"); keys and values share one selection (caption of the paper's main table).
+ *   Kc[offsets[u] + t, :] = K[unit u, indices[offsets[u] + t], :]   for t < offsets[u+1] - offsets[u]
+ * and the same for V.  Rows are copied bit for bit.
+ *
+ * d_K, d_V    in   [B, L, H, N, d] with strides sK, sV
+ * d_indices   in   [offsets[units]] int32
+ * d_offsets   in   [B*L*H + 1] int64
+ * d_Kc, d_Vc  out  [offsets[units], d] contiguous, storage dtype, 16-byte aligned
+ * ------------------------------------------------------------------------------------------------- */
+int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_strides sK, uncomp_strides sV,
+                   const int32_t *d_indices, const int64_t *d_offsets, void *d_Kc, void *d_Vc, void *stream);
+
+/* Synchronise `stream`, copy the status word to *host_bits and clear it on the device.  The only call
+ * that waits for the device. */
+int uncomp_status(uncomp_ctx *ctx, void *stream, uint32_t *host_bits);
+
+/* Text for a return code; never NULL. */
+const char *uncomp_strerror(int code);
+
+/* The cudaError_t (as int) behind the most recent UNCOMP_E_CUDA of this context, else 0. */
+int uncomp_last_cuda_error(const uncomp_ctx *ctx);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int uncomp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UNCOMP_H_ */

@@ -1,0 +1,233 @@
+// Host side of the C ABI declared in include/uncomp.h: argument checks, the workspace plan and the
+// kernel launches of the four calls.  No device memory is allocated here.
+#include <math.h>
+#include <new>
+
+#include "common.cuh"
+
+namespace uncomp {
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static bool shape_ok(const uncomp_shape &s) {
+    if (s.B < 1 || s.L < 1 || s.H < 1 || s.Hq < 1 || s.N < 2) return false;
+    if (s.d != kD) return false;
+    if (s.Hq % s.H != 0) return false;
+    if (s.w < 1 || s.w > 64 || s.w >= s.N) return false;
+    if ((s.Hq / s.H) * s.w > kMaxRows) return false;
+    if (s.dtype != UNCOMP_BF16 && s.dtype != UNCOMP_FP32) return false;
+    if ((int64_t)s.B * s.L * s.H > (1 << 20)) return false;
+    if (s.N > (1 << 24)) return false;
+    return true;
+}
+
+Plan make_plan(const uncomp_shape &s) {
+    Plan p;
+    p.shape = s;
+    p.units = s.B * s.L * s.H;
+    p.G = s.Hq / s.H;
+    p.rows = p.G * s.w;
+    p.prefix = s.N - s.w;
+    const int target_ctas = 592;   // four CTAs for each of the 148 SMs
+    {
+        int want = (target_ctas + p.units - 1) / p.units;
+        int most = (s.N + 1023) / 1024;
+        int P = want < 1 ? 1 : (want > most ? most : want);
+        int chunk = (int)align_up((size_t)(s.N + P - 1) / P, 128);
+        p.gram_chunk = chunk;
+        p.gram_splits = (s.N + chunk - 1) / chunk;
+    }
+    {
+        int want = (target_ctas + p.units - 1) / p.units;
+        int most = (s.N + 511) / 512;
+        int P = want < 1 ? 1 : (want > most ? most : want);
+        int chunk = (int)align_up((size_t)(s.N + P - 1) / P, 64);
+        p.score_chunk = chunk;
+        p.score_splits = (s.N + chunk - 1) / chunk;
+    }
+    const size_t acc = s.dtype == UNCOMP_FP32 ? sizeof(double) : sizeof(float);
+    size_t o = 0;
+    p.off_status = o;      o = align_up(o + 256, 256);
+    p.off_gram = o;        o = align_up(o + (size_t)p.units * p.gram_splits * (kD * kD + kD) * acc, 256);
+    p.off_stats_part = o;  o = align_up(o + (size_t)p.units * p.score_splits * kMaxRows * 2 * sizeof(float), 256);
+    p.off_stats = o;       o = align_up(o + (size_t)p.units * kMaxRows * 2 * sizeof(float), 256);
+    p.off_raw = o;         o = align_up(o + (size_t)p.units * p.prefix * sizeof(float), 256);
+    p.off_pooled = o;      o = align_up(o + (size_t)p.units * p.prefix * sizeof(float), 256);
+    p.off_rank = o;        o = align_up(o + (size_t)p.units * sizeof(int32_t), 256);
+    p.off_rem = o;         o = align_up(o + (size_t)p.units * sizeof(int64_t), 256);
+    p.bytes = o;
+    return p;
+}
+
+}  // namespace uncomp
+
+using namespace uncomp;
+
+struct uncomp_ctx {
+    Plan plan;
+    unsigned char *ws;
+    int last_cuda;
+    int device;
+};
+
+static int cuda_fail(uncomp_ctx *ctx, cudaError_t e) {
+    ctx->last_cuda = (int)e;
+    return UNCOMP_E_CUDA;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_strides(const uncomp_shape &s, const uncomp_strides &st) {
+    const int64_t eb = s.dtype == UNCOMP_FP32 ? 4 : 2;
+    const int64_t v[4] = {st.sB, st.sL, st.sH, st.sN};
+    for (int i = 0; i < 4; ++i) {
+        if (v[i] < 0) return UNCOMP_E_SHAPE;
+        if ((v[i] * eb) % 16 != 0) return UNCOMP_E_ALIGN;
+    }
+    if (st.sN < s.d) return UNCOMP_E_SHAPE;
+    return UNCOMP_OK;
+}
+
+extern "C" {
+
+int uncomp_version(void) { return 100; }
+
+const char *uncomp_strerror(int code) {
+    switch (code) {
+        case UNCOMP_OK: return "ok";
+        case UNCOMP_E_NULL: return "a required pointer is NULL";
+        case UNCOMP_E_SHAPE: return "unsupported shape or stride";
+        case UNCOMP_E_ALIGN: return "pointer or stride is not 16-byte aligned";
+        case UNCOMP_E_WORKSPACE: return "workspace too small or misaligned";
+        case UNCOMP_E_PARAM: return "invalid hyper-parameter";
+        case UNCOMP_E_CUDA: return "CUDA call failed";
+        case UNCOMP_E_LIMIT: return "size beyond a documented maximum";
+        default: return "unknown error code";
+    }
+}
+
+size_t uncomp_workspace_bytes(const uncomp_shape *shape) {
+    if (!shape || !shape_ok(*shape)) return 0;
+    return make_plan(*shape).bytes;
+}
+
+int uncomp_create(uncomp_ctx **out, const uncomp_shape *shape, void *d_workspace, size_t workspace_bytes) {
+    if (!out || !shape || !d_workspace) return UNCOMP_E_NULL;
+    *out = nullptr;
+    if (!shape_ok(*shape)) return UNCOMP_E_SHAPE;
+    Plan p = make_plan(*shape);
+    if (workspace_bytes < p.bytes || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return UNCOMP_E_WORKSPACE;
+    uncomp_ctx *ctx = new (std::nothrow) uncomp_ctx;
+    if (!ctx) return UNCOMP_E_LIMIT;
+    ctx->plan = p;
+    ctx->ws = static_cast<unsigned char *>(d_workspace);
+    ctx->last_cuda = 0;
+    ctx->device = 0;
+    cudaError_t e = cudaGetDevice(&ctx->device);
+    if (e == cudaSuccess) e = cudaMemset(ctx->ws + p.off_status, 0, 256);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        delete ctx;
+        return UNCOMP_E_CUDA;
+    }
+    *out = ctx;
+    return UNCOMP_OK;
+}
+
+void uncomp_destroy(uncomp_ctx *ctx) { delete ctx; }
+
+int uncomp_last_cuda_error(const uncomp_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const uncomp_entropy_params *params,
+                   float *d_entropy, float *d_erank, double *d_spectrum, void *stream) {
+    if (!ctx || !d_K || !params || !d_entropy) return UNCOMP_E_NULL;
+    const Plan &p = ctx->plan;
+    if (!aligned16(d_K)) return UNCOMP_E_ALIGN;
+    int rc = check_strides(p.shape, sK);
+    if (rc != UNCOMP_OK) return rc;
+    if (params->k_trunc < 1 || params->max_iters < 0 || (params->center != 0 && params->center != 1) ||
+        (params->norm != 0 && params->norm != 1))
+        return UNCOMP_E_PARAM;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t *d_status = reinterpret_cast<uint32_t *>(ctx->ws + p.off_status);
+    void *partials = ctx->ws + p.off_gram;
+    const UnitAddr addr = make_addr(p.shape, sK);
+    cudaError_t e = launch_gram_simt(p, d_K, addr, partials, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = launch_eigen_entropy(p, partials, *params, d_entropy, d_erank, d_spectrum, d_status, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+int uncomp_assign_budgets(uncomp_ctx *ctx, const float *d_erank, const uncomp_budget_params *params,
+                          int32_t *d_budgets, int64_t *d_offsets, int32_t *d_layer_group,
+                          int32_t *d_layer_ctx, void *stream) {
+    if (!ctx || !d_erank || !params || !d_budgets || !d_offsets) return UNCOMP_E_NULL;
+    const Plan &p = ctx->plan;
+    if (params->scope != 0 && params->scope != 1) return UNCOMP_E_PARAM;
+    const int rc = check_budget_params(p.shape, *params);
+    if (rc != UNCOMP_OK) return rc;
+    if ((d_layer_group == nullptr) != (d_layer_ctx == nullptr)) return UNCOMP_E_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_budgets(p, d_erank, *params, d_budgets, d_offsets, d_layer_group, d_layer_ctx,
+                                   reinterpret_cast<int32_t *>(ctx->ws + p.off_rank),
+                                   reinterpret_cast<int64_t *>(ctx->ws + p.off_rem), st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, uncomp_strides sK,
+                        const int32_t *d_budgets, const int64_t *d_offsets, const uncomp_score_params *params,
+                        float *d_scores, int32_t *d_indices, void *stream) {
+    if (!ctx || !d_Qw || !d_K || !d_budgets || !d_offsets || !params || !d_indices) return UNCOMP_E_NULL;
+    const Plan &p = ctx->plan;
+    if (!aligned16(d_K) || !aligned16(d_Qw)) return UNCOMP_E_ALIGN;
+    int rc = check_strides(p.shape, sK);
+    if (rc != UNCOMP_OK) return rc;
+    if (params->pool_kernel < 1 || params->pool_kernel > 63 || (params->pool_kernel & 1) == 0 ||
+        (params->pool_mode != 0 && params->pool_mode != 1) || !(params->scale >= 0.f) || isinf(params->scale))
+        return UNCOMP_E_PARAM;
+    const float scale = params->scale > 0.f ? params->scale : 1.0f / sqrtf((float)p.shape.d);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t *d_status = reinterpret_cast<uint32_t *>(ctx->ws + p.off_status);
+    float *stats_part = reinterpret_cast<float *>(ctx->ws + p.off_stats_part);
+    float *stats = reinterpret_cast<float *>(ctx->ws + p.off_stats);
+    float *raw = reinterpret_cast<float *>(ctx->ws + p.off_raw);
+    float *pooled = d_scores ? d_scores : reinterpret_cast<float *>(ctx->ws + p.off_pooled);
+    const UnitAddr addr = make_addr(p.shape, sK);
+    cudaError_t e = launch_scores_simt(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = launch_pool_select(p, raw, pooled, params->pool_kernel, params->pool_mode, d_budgets, d_offsets, d_indices,
+                           d_status, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_strides sK, uncomp_strides sV,
+                   const int32_t *d_indices, const int64_t *d_offsets, void *d_Kc, void *d_Vc, void *stream) {
+    if (!ctx || !d_K || !d_V || !d_indices || !d_offsets || !d_Kc || !d_Vc) return UNCOMP_E_NULL;
+    const Plan &p = ctx->plan;
+    if (!aligned16(d_K) || !aligned16(d_V) || !aligned16(d_Kc) || !aligned16(d_Vc)) return UNCOMP_E_ALIGN;
+    int rc = check_strides(p.shape, sK);
+    if (rc != UNCOMP_OK) return rc;
+    rc = check_strides(p.shape, sV);
+    if (rc != UNCOMP_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_compact(p, d_K, d_V, make_addr(p.shape, sK), make_addr(p.shape, sV), d_indices,
+                                   d_offsets, d_Kc, d_Vc, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+int uncomp_status(uncomp_ctx *ctx, void *stream, uint32_t *host_bits) {
+    if (!ctx || !host_bits) return UNCOMP_E_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t *d_status = reinterpret_cast<uint32_t *>(ctx->ws + ctx->plan.off_status);
+    cudaError_t e = cudaMemcpyAsync(host_bits, d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(d_status, 0, sizeof(uint32_t), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,79 @@
+// Shared device/host helpers of the uncomp CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/uncomp.h"
+
+namespace uncomp {
+
+constexpr int kD = 128;          // head dimension supported by every kernel
+constexpr int kMaxRows = 512;    // G * w upper bound (window rows of all grouped query heads)
+
+// Carve-up of the caller's workspace, decided by the shape alone (see api.cu).
+struct Plan {
+    uncomp_shape shape;
+    int units;          // B * L * H
+    int G;              // query heads per KV head
+    int rows;           // G * w
+    int prefix;         // N - w
+    int gram_splits;    // token chunks per unit in the Gram stage (P)
+    int gram_chunk;     // tokens per chunk
+    int score_splits;   // token chunks per unit in the scorer's statistics pass
+    int score_chunk;    // tokens per chunk
+    size_t off_status, off_gram, off_stats_part, off_stats, off_raw, off_pooled, off_rank, off_rem;
+    size_t bytes;
+};
+
+struct UnitAddr {
+    int L, H;
+    int64_t sB, sL, sH, sN;
+    __host__ __device__ inline int64_t base(int u) const {
+        const int h = u % H;
+        const int l = (u / H) % L;
+        const int b = u / (H * L);
+        return (int64_t)b * sB + (int64_t)l * sL + (int64_t)h * sH;
+    }
+};
+
+inline UnitAddr make_addr(const uncomp_shape &s, const uncomp_strides &st) {
+    UnitAddr a;
+    a.L = s.L; a.H = s.H; a.sB = st.sB; a.sL = st.sL; a.sH = st.sH; a.sN = st.sN;
+    return a;
+}
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ---- kernel launchers (each returns the cudaError_t of its launches) -------------------------------
+cudaError_t launch_gram_simt(const Plan &p, const void *dK, const UnitAddr &addr, void *d_partials, cudaStream_t st);
+cudaError_t launch_eigen_entropy(const Plan &p, const void *d_partials, const uncomp_entropy_params &ep,
+                                 float *d_entropy, float *d_erank, double *d_spectrum, uint32_t *d_status,
+                                 cudaStream_t st);
+int check_budget_params(const uncomp_shape &s, const uncomp_budget_params &bp);
+cudaError_t launch_budgets(const Plan &p, const float *d_erank, const uncomp_budget_params &bp, int32_t *d_budgets,
+                           int64_t *d_offsets, int32_t *d_layer_group, int32_t *d_layer_ctx, int32_t *d_rank,
+                           int64_t *d_rem, cudaStream_t st);
+cudaError_t launch_scores_simt(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
+                               float *d_stats_part, float *d_stats, float *d_raw, cudaStream_t st);
+cudaError_t launch_pool_select(const Plan &p, const float *d_raw, float *d_pooled, int pool_kernel, int pool_mode,
+                               const int32_t *d_budgets, const int64_t *d_offsets, int32_t *d_indices,
+                               uint32_t *d_status, cudaStream_t st);
+cudaError_t launch_compact(const Plan &p, const void *dK, const void *dV, const UnitAddr &aK, const UnitAddr &aV,
+                           const int32_t *d_indices, const int64_t *d_offsets, void *dKc, void *dVc,
+                           cudaStream_t st);
+
+}  // namespace uncomp

@@ -1,0 +1,153 @@
+// Pooling of the raw window scores and variable-k top-k selection per unit (paper Section 3.3.3:
+// the tokens with the highest cumulative window attention are kept within the head's budget; the w
+// window tokens are part of the budget).
+//
+// One CTA of 1024 threads per unit.
+//   1. pooled[j] = max / mean of raw over the pool window clipped to the prefix (written out: it is the
+//      `d_scores` output of the pass).
+//   2. Radix select of the k-th largest pooled score, k = budget - w, on the order-preserving 32-bit
+//      image of the float: three histogram passes (11 + 11 + 10 bits) give the exact threshold T, the
+//      number of scores above it and how many scores equal to T are still needed.
+//   3. Ordered compaction: each warp owns a contiguous segment; ballots and population counts give every
+//      kept position its output slot, so the kept positions come out ascending, and among scores equal to
+//      T the lowest positions win.  The window positions follow.
+// Counting is integer work: the result does not depend on the order in which threads run.
+#include "common.cuh"
+
+namespace uncomp {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+
+__device__ __forceinline__ uint32_t ordered_bits(float f) {
+    const uint32_t b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+struct SelSmem {
+    int hist[2048];
+    int scan[kSelThreads];
+    int warp_gt[kSelWarps], warp_eq[kSelWarps];
+    int bin, above;
+};
+
+// Finds the bin (counting down from the top) that holds the kr-th largest element.  All threads call it.
+__device__ void find_bin(SelSmem &S, int nbins, int kr, int tid) {
+    // thread t covers bins nbins-1-2t and nbins-2-2t
+    const int b0 = nbins - 1 - 2 * tid;
+    const int h0 = b0 >= 0 ? S.hist[b0] : 0;
+    const int h1 = b0 - 1 >= 0 ? S.hist[b0 - 1] : 0;
+    S.scan[tid] = h0 + h1;
+    __syncthreads();
+    for (int o = 1; o < kSelThreads; o <<= 1) {
+        const int add = tid >= o ? S.scan[tid - o] : 0;
+        __syncthreads();
+        S.scan[tid] += add;
+        __syncthreads();
+    }
+    const int excl = S.scan[tid] - (h0 + h1);
+    if (b0 >= 0 && excl < kr && kr <= excl + h0) { S.bin = b0; S.above = excl; }
+    else if (b0 - 1 >= 0 && excl + h0 < kr && kr <= excl + h0 + h1) { S.bin = b0 - 1; S.above = excl + h0; }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float *__restrict__ raw,
+                                                                 float *__restrict__ pooled, int P, int w,
+                                                                 int pool_kernel, int pool_mode,
+                                                                 const int32_t *__restrict__ budgets,
+                                                                 const int64_t *__restrict__ offsets,
+                                                                 int32_t *__restrict__ indices,
+                                                                 uint32_t *__restrict__ status) {
+    __shared__ SelSmem S;
+    const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const float *r = raw + (size_t)u * P;
+    float *s = pooled + (size_t)u * P;
+
+    // ---- 1. pooling ------------------------------------------------------------------------------
+    const int half = pool_kernel >> 1;
+    for (int j = tid; j < P; j += kSelThreads) {
+        const int lo = max(0, j - half), hi = min(P - 1, j + half);
+        float acc = pool_mode ? 0.f : r[lo];
+        for (int t = lo; t <= hi; ++t) acc = pool_mode ? acc + r[t] : fmaxf(acc, r[t]);
+        s[j] = pool_mode ? acc / (float)(hi - lo + 1) : acc;
+    }
+    int budget = budgets[u];
+    if (budget < w || budget > P + w) {
+        if (tid == 0) atomicOr(status, UNCOMP_STATUS_BOUNDS);
+        budget = min(max(budget, w), P + w);
+    }
+    const int k = budget - w;
+    int32_t *out = indices + offsets[u];
+    for (int i = tid; i < w; i += kSelThreads) out[k + i] = P + i;
+    if (k == 0) return;   // uniform over the CTA
+    __syncthreads();      // pooled scores of this unit are visible to the whole CTA
+
+    // ---- 2. threshold ----------------------------------------------------------------------------
+    uint32_t prefix = 0;      // bits of the threshold fixed so far
+    int kr = k;               // rank still to resolve inside the current bin
+    if (k < P) {
+#pragma unroll 1
+        for (int pass = 0; pass < 3; ++pass) {
+            const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+            const int nbits = pass == 2 ? 10 : 11;
+            const int nbins = 1 << nbits;
+            const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + nbits));
+            for (int b = tid; b < 2048; b += kSelThreads) S.hist[b] = 0;
+            __syncthreads();
+            for (int j = tid; j < P; j += kSelThreads) {
+                const uint32_t v = ordered_bits(s[j]);
+                if ((v & himask) == prefix) atomicAdd(&S.hist[(v >> shift) & (nbins - 1)], 1);
+            }
+            __syncthreads();
+            find_bin(S, nbins, kr, tid);
+            prefix |= (uint32_t)S.bin << shift;
+            kr -= S.above;
+            __syncthreads();
+        }
+    }
+    // k >= P keeps every prefix position: threshold below everything
+    const uint32_t T = k < P ? prefix : 0u;
+    const int need_eq = k < P ? kr : P;   // scores equal to T that are still kept (lowest positions first)
+
+    // ---- 3. ordered compaction -------------------------------------------------------------------
+    const int seg = ((P + kSelWarps - 1) / kSelWarps + 31) & ~31;
+    const int j0 = min(P, wid * seg), j1 = min(P, j0 + seg);
+    int cg = 0, ce = 0;
+    for (int j = j0 + lane; j < j1; j += 32) {
+        const uint32_t v = ordered_bits(s[j]);
+        cg += v > T;
+        ce += v == T;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        cg += __shfl_xor_sync(0xffffffffu, cg, o);
+        ce += __shfl_xor_sync(0xffffffffu, ce, o);
+    }
+    if (lane == 0) { S.warp_gt[wid] = cg; S.warp_eq[wid] = ce; }
+    __syncthreads();
+    int gt_run = 0, eq_run = 0;
+    for (int x = 0; x < wid; ++x) { gt_run += S.warp_gt[x]; eq_run += S.warp_eq[x]; }
+    const unsigned lt = (1u << lane) - 1u;
+    for (int jb = j0; jb < j1; jb += 32) {
+        const int j = jb + lane;
+        const uint32_t v = j < j1 ? ordered_bits(s[j]) : 0u;
+        const bool gt = j < j1 && v > T;
+        const bool eq = j < j1 && v == T;
+        const unsigned mg = __ballot_sync(0xffffffffu, gt), me = __ballot_sync(0xffffffffu, eq);
+        const int gtb = gt_run + __popc(mg & lt);
+        const int eqb = eq_run + __popc(me & lt);
+        if (gt || (eq && eqb < need_eq)) out[gtb + min(eqb, need_eq)] = j;
+        gt_run += __popc(mg);
+        eq_run += __popc(me);
+    }
+}
+
+cudaError_t launch_pool_select(const Plan &p, const float *d_raw, float *d_pooled, int pool_kernel, int pool_mode,
+                               const int32_t *d_budgets, const int64_t *d_offsets, int32_t *d_indices,
+                               uint32_t *d_status, cudaStream_t st) {
+    pool_select_kernel<<<p.units, kSelThreads, 0, st>>>(d_raw, d_pooled, p.prefix, p.shape.w, pool_kernel, pool_mode,
+                                                        d_budgets, d_offsets, d_indices, d_status);
+    return cudaGetLastError();
+}
+
+}  // namespace uncomp
