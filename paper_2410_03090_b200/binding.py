@@ -1,0 +1,206 @@
+"""Thin ctypes binding over libuncomp.so: the same names as include/uncomp.h, argument marshalling only.
+
+Every step of the pass runs in the CUDA library.  PyTorch supplies device memory and streams.  There is
+no CPU fallback: if the library cannot be loaded, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+UNCOMP_BF16, UNCOMP_FP32 = 0, 1
+UNCOMP_OK = 0
+UNCOMP_E_NULL, UNCOMP_E_SHAPE, UNCOMP_E_ALIGN, UNCOMP_E_WORKSPACE = -1, -2, -3, -4
+UNCOMP_E_PARAM, UNCOMP_E_CUDA, UNCOMP_E_LIMIT = -5, -6, -7
+UNCOMP_STATUS_NOT_CONVERGED, UNCOMP_STATUS_TIMEOUT, UNCOMP_STATUS_BOUNDS = 1, 2, 4
+
+
+class uncomp_shape(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("B", "L", "H", "Hq", "N", "d", "w", "dtype")]
+
+
+class uncomp_strides(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("sB", "sL", "sH", "sN")]
+
+
+class uncomp_entropy_params(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("k_trunc", "center", "norm", "max_iters")]
+
+
+class uncomp_budget_params(C.Structure):
+    _fields_ = [("avg_budget", C.c_int32), ("M", C.c_int32), ("n_max", C.c_int32), ("scope", C.c_int32),
+                ("eps", C.c_float), ("dn", C.c_int32), ("n_last", C.c_int32)]
+
+
+class uncomp_score_params(C.Structure):
+    _fields_ = [("pool_kernel", C.c_int32), ("pool_mode", C.c_int32), ("scale", C.c_float)]
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()
+    lib = C.CDLL(path)
+    vp, i32p, i64p, fp, dp = C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p
+    lib.uncomp_version.restype = C.c_int
+    lib.uncomp_strerror.restype = C.c_char_p
+    lib.uncomp_strerror.argtypes = [C.c_int]
+    lib.uncomp_workspace_bytes.restype = C.c_size_t
+    lib.uncomp_workspace_bytes.argtypes = [C.POINTER(uncomp_shape)]
+    lib.uncomp_create.restype = C.c_int
+    lib.uncomp_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(uncomp_shape), vp, C.c_size_t]
+    lib.uncomp_destroy.restype = None
+    lib.uncomp_destroy.argtypes = [vp]
+    lib.uncomp_last_cuda_error.restype = C.c_int
+    lib.uncomp_last_cuda_error.argtypes = [vp]
+    lib.uncomp_entropy.restype = C.c_int
+    lib.uncomp_entropy.argtypes = [vp, vp, uncomp_strides, C.POINTER(uncomp_entropy_params), fp, fp, dp, vp]
+    lib.uncomp_assign_budgets.restype = C.c_int
+    lib.uncomp_assign_budgets.argtypes = [vp, fp, C.POINTER(uncomp_budget_params), i32p, i64p, i32p, i32p, vp]
+    lib.uncomp_score_select.restype = C.c_int
+    lib.uncomp_score_select.argtypes = [vp, vp, vp, uncomp_strides, i32p, i64p, C.POINTER(uncomp_score_params),
+                                        fp, i32p, vp]
+    lib.uncomp_compact.restype = C.c_int
+    lib.uncomp_compact.argtypes = [vp, vp, vp, uncomp_strides, uncomp_strides, i32p, i64p, vp, vp, vp]
+    lib.uncomp_status.restype = C.c_int
+    lib.uncomp_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
+    return lib
+
+
+lib = _load()
+
+
+class UncompError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {lib.uncomp_strerror(code).decode()} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != UNCOMP_OK:
+        raise UncompError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream: Optional[torch.cuda.Stream]):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def make_shape(B, L, H, Hq, N, d, w, dtype) -> uncomp_shape:
+    code = {torch.bfloat16: UNCOMP_BF16, torch.float32: UNCOMP_FP32, "bf16": UNCOMP_BF16, "fp32": UNCOMP_FP32}[dtype]
+    return uncomp_shape(B, L, H, Hq, N, d, w, code)
+
+
+def strides_of(t: torch.Tensor) -> uncomp_strides:
+    """Element strides of a [B, L, H, N, d] tensor (d contiguous)."""
+    if t.dim() != 5 or t.stride(4) != 1:
+        raise ValueError("expected a [B, L, H, N, d] tensor with a contiguous last dimension")
+    return uncomp_strides(t.stride(0), t.stride(1), t.stride(2), t.stride(3))
+
+
+def uncomp_workspace_bytes(shape: uncomp_shape) -> int:
+    return int(lib.uncomp_workspace_bytes(C.byref(shape)))
+
+
+class Context:
+    """uncomp_ctx plus the torch tensor that backs its workspace."""
+
+    def __init__(self, shape: uncomp_shape, device: torch.device | str = "cuda"):
+        self.shape = shape
+        nbytes = uncomp_workspace_bytes(shape)
+        if nbytes == 0:
+            raise UncompError(UNCOMP_E_SHAPE, "uncomp_workspace_bytes")
+        self.device = torch.device(device)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + 255) // 256 * 256
+        self.workspace_bytes = nbytes
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(lib.uncomp_create(C.byref(h), C.byref(shape), C.c_void_p(self._ws_ptr), nbytes), "uncomp_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib.uncomp_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def uncomp_entropy(ctx: Context, K: torch.Tensor, k_trunc: int = 32, center: int = 1, norm: int = 0,
+                   max_iters: int = 0, entropy: Optional[torch.Tensor] = None, erank: Optional[torch.Tensor] = None,
+                   spectrum: Optional[torch.Tensor] = None, stream=None):
+    s = ctx.shape
+    if entropy is None:
+        entropy = torch.empty(s.B, s.L, s.H, dtype=torch.float32, device=K.device)
+    if erank is None:
+        erank = torch.empty(s.B, s.L, s.H, dtype=torch.float32, device=K.device)
+    p = uncomp_entropy_params(k_trunc, center, norm, max_iters)
+    _check(lib.uncomp_entropy(ctx.handle, _ptr(K), strides_of(K), C.byref(p), _ptr(entropy), _ptr(erank),
+                              _ptr(spectrum), _stream(stream)), "uncomp_entropy")
+    return entropy, erank
+
+
+def uncomp_assign_budgets(ctx: Context, erank: torch.Tensor, avg_budget: int, M: int, n_max: int, scope: int = 0,
+                          eps: float = 0.0, dn: int = 0, n_last: int = 0, budgets=None, offsets=None,
+                          layer_group=None, layer_ctx=None, stream=None):
+    s = ctx.shape
+    dev = erank.device
+    units = s.B * s.L * s.H
+    if budgets is None:
+        budgets = torch.empty(s.B, s.L, s.H, dtype=torch.int32, device=dev)
+    if offsets is None:
+        offsets = torch.empty(units + 1, dtype=torch.int64, device=dev)
+    if layer_group is None:
+        layer_group = torch.empty(s.B, s.L, dtype=torch.int32, device=dev)
+    if layer_ctx is None:
+        layer_ctx = torch.empty(s.B, s.L, dtype=torch.int32, device=dev)
+    p = uncomp_budget_params(avg_budget, M, n_max, scope, eps, dn, n_last)
+    _check(lib.uncomp_assign_budgets(ctx.handle, _ptr(erank), C.byref(p), _ptr(budgets), _ptr(offsets),
+                                     _ptr(layer_group), _ptr(layer_ctx), _stream(stream)), "uncomp_assign_budgets")
+    return budgets, offsets, layer_group, layer_ctx
+
+
+def uncomp_score_select(ctx: Context, Qw: torch.Tensor, K: torch.Tensor, budgets: torch.Tensor,
+                        offsets: torch.Tensor, total_rows: int, pool_kernel: int = 7, pool_mode: int = 0,
+                        scale: float = 0.0, scores: Optional[torch.Tensor] = None,
+                        indices: Optional[torch.Tensor] = None, stream=None):
+    if indices is None:
+        indices = torch.empty(total_rows, dtype=torch.int32, device=K.device)
+    p = uncomp_score_params(pool_kernel, pool_mode, scale)
+    _check(lib.uncomp_score_select(ctx.handle, _ptr(Qw), _ptr(K), strides_of(K), _ptr(budgets), _ptr(offsets),
+                                   C.byref(p), _ptr(scores), _ptr(indices), _stream(stream)), "uncomp_score_select")
+    return indices
+
+
+def uncomp_compact(ctx: Context, K: torch.Tensor, V: torch.Tensor, indices: torch.Tensor, offsets: torch.Tensor,
+                   total_rows: int, Kc: Optional[torch.Tensor] = None, Vc: Optional[torch.Tensor] = None, stream=None):
+    d = ctx.shape.d
+    if Kc is None:
+        Kc = torch.empty(total_rows, d, dtype=K.dtype, device=K.device)
+    if Vc is None:
+        Vc = torch.empty(total_rows, d, dtype=V.dtype, device=V.device)
+    _check(lib.uncomp_compact(ctx.handle, _ptr(K), _ptr(V), strides_of(K), strides_of(V), _ptr(indices),
+                              _ptr(offsets), _ptr(Kc), _ptr(Vc), _stream(stream)), "uncomp_compact")
+    return Kc, Vc
+
+
+def uncomp_status(ctx: Context, stream=None) -> int:
+    bits = C.c_uint32(0)
+    _check(lib.uncomp_status(ctx.handle, _stream(stream), C.byref(bits)), "uncomp_status")
+    return int(bits.value)

@@ -1,0 +1,62 @@
+"""The whole compression pass as one call: the four C-ABI calls back to back on one stream."""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import binding as ub
+from .synth import Workload
+
+
+@dataclass
+class PassOutput:
+    entropy: torch.Tensor      # [B, L, H] float32, H_k
+    erank: torch.Tensor        # [B, L, H] float32, erank_k
+    budgets: torch.Tensor      # [B, L, H] int32
+    offsets: torch.Tensor      # [units + 1] int64
+    layer_group: torch.Tensor  # [B, L] int32
+    layer_ctx: torch.Tensor    # [B, L] int32
+    scores: torch.Tensor       # [B, L, H, N - w] float32, pooled window scores
+    indices: torch.Tensor      # [total_rows] int32
+    Kc: torch.Tensor           # [total_rows, d]
+    Vc: torch.Tensor           # [total_rows, d]
+
+
+class CompressionPass:
+    """Pre-allocates every output of a workload once; `run` launches the pass without host syncs."""
+
+    def __init__(self, wl: Workload, device: torch.device | str = "cuda"):
+        self.wl = wl
+        self.device = torch.device(device)
+        self.shape = ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype)
+        self.ctx = ub.Context(self.shape, self.device)
+        dev, u = self.device, wl.units
+        f32, i32 = torch.float32, torch.int32
+        self.out = PassOutput(
+            entropy=torch.empty(wl.B, wl.L, wl.H, dtype=f32, device=dev),
+            erank=torch.empty(wl.B, wl.L, wl.H, dtype=f32, device=dev),
+            budgets=torch.empty(wl.B, wl.L, wl.H, dtype=i32, device=dev),
+            offsets=torch.empty(u + 1, dtype=torch.int64, device=dev),
+            layer_group=torch.empty(wl.B, wl.L, dtype=i32, device=dev),
+            layer_ctx=torch.empty(wl.B, wl.L, dtype=i32, device=dev),
+            scores=torch.empty(wl.B, wl.L, wl.H, wl.N - wl.w, dtype=f32, device=dev),
+            indices=torch.empty(wl.total_rows, dtype=i32, device=dev),
+            Kc=torch.empty(wl.total_rows, wl.d, dtype=wl.torch_dtype, device=dev),
+            Vc=torch.empty(wl.total_rows, wl.d, dtype=wl.torch_dtype, device=dev),
+        )
+
+    def run(self, K: torch.Tensor, V: torch.Tensor, Qw: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
+            eps: float = 0.0, dn: int = 0, n_last: int = 0, scope: int = 0) -> PassOutput:
+        wl, o, ctx = self.wl, self.out, self.ctx
+        ub.uncomp_entropy(ctx, K, wl.k_trunc, 1, 0, 0, o.entropy, o.erank, None, stream)
+        ub.uncomp_assign_budgets(ctx, o.erank, wl.avg_budget, wl.M, wl.n_max, scope, eps, dn, n_last,
+                                 o.budgets, o.offsets, o.layer_group, o.layer_ctx, stream)
+        ub.uncomp_score_select(ctx, Qw, K, o.budgets, o.offsets, wl.total_rows, wl.pool_kernel, wl.pool_mode, 0.0,
+                               o.scores, o.indices, stream)
+        ub.uncomp_compact(ctx, K, V, o.indices, o.offsets, wl.total_rows, o.Kc, o.Vc, stream)
+        return o
+
+    def status(self, stream=None) -> int:
+        return ub.uncomp_status(self.ctx, stream)

@@ -1,0 +1,249 @@
+"""Parity of the CUDA library against the CPU oracle, stage by stage, through the C ABI.
+
+Tolerances (written out in tests/parity.py): entropies 1e-4 relative (floor |H| = 1), window scores 2e-3
+relative; budgets, selected indices and compacted rows bit-exact under the stage protocol (the oracle's
+rule applied to the GPU's own erank / pooled scores)."""
+import numpy as np
+import pytest
+import torch
+
+import parity
+from paper_2410_03090_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _ub():
+    from paper_2410_03090_b200 import binding
+    return binding
+
+
+def _run(wl, **kw):
+    from paper_2410_03090_b200.compress import CompressionPass
+    K, V, Qw = synth.generate(wl, "cuda")
+    cp = CompressionPass(wl, "cuda")
+    out = cp.run(K, V, Qw, **kw)
+    torch.cuda.synchronize()
+    assert cp.status() == 0
+    return K, V, Qw, cp, out
+
+
+def _check_all(wl, K, V, Qw, out, units, **bkw):
+    parity.check_entropy(wl, K, out.entropy, out.erank, units)
+    parity.check_budgets(wl, out.erank, out.budgets, out.offsets, out.layer_group, out.layer_ctx, **bkw)
+    parity.check_scores(wl, K, Qw, out.scores, units)
+    parity.check_select(wl, out.scores, out.budgets, out.offsets, out.indices, range(wl.units))
+    parity.check_compact(wl, K, V, out.indices, out.offsets, out.Kc, out.Vc, units)
+    assert int(out.offsets[-1]) == wl.total_rows
+
+
+def test_config1_fp32_whole_pass():
+    wl = synth.WORKLOADS["c1"]
+    K, V, Qw, cp, out = _run(wl)
+    _check_all(wl, K, V, Qw, out, range(wl.units))
+
+
+@pytest.mark.parametrize("name,N,L", [("c2", 1000, 2), ("c3", 2309, 8), ("c5", 1536, 1)])
+def test_bf16_small_whole_pass(name, N, L):
+    # several token tiles and a ragged tail; c3 includes its near-isotropic head, c5 has G = 8, w = 64
+    wl = synth.scaled(synth.WORKLOADS[name], N=N, L=L)
+    K, V, Qw, cp, out = _run(wl, eps=0.3, dn=256, n_last=512)
+    _check_all(wl, K, V, Qw, out, range(0, wl.units, 3), eps=0.3, dn=256, n_last=512)
+
+
+def test_c4_batch_with_norm_spikes():
+    wl = synth.scaled(synth.WORKLOADS["c4"], N=1280, L=1, B=2)
+    K, V, Qw, cp, out = _run(wl)
+    _check_all(wl, K, V, Qw, out, range(0, wl.units, 2))
+
+
+def test_spectrum_matches_oracle_eigenvalues():
+    import oracle
+    ub = _ub()
+    wl = synth.WORKLOADS["c1"]
+    K, _, _ = synth.generate(wl, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    spec = torch.empty(wl.B, wl.L, wl.H, 128, dtype=torch.float64, device="cuda")
+    ent, er = ub.uncomp_entropy(ctx, K, k_trunc=128, norm=1, spectrum=spec)
+    torch.cuda.synchronize()
+    for u in range(wl.units):
+        H, E, lam = oracle.entropy(parity.unit_np(K, wl, u), k_trunc=128, norm=1, return_spectrum=True)
+        got = spec.reshape(-1, 128)[u].cpu().numpy()
+        np.testing.assert_allclose(got, lam, rtol=0, atol=1e-11 * lam[0])
+        assert abs(float(ent.reshape(-1)[u]) - H) <= 1e-4 * max(abs(H), 1.0)
+
+
+@pytest.mark.parametrize("k_trunc,center,norm", [(16, 1, 0), (64, 0, 0), (32, 1, 1), (200, 0, 1)])
+def test_entropy_variants(k_trunc, center, norm):
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=777, L=1)
+    K, _, _ = synth.generate(wl, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    ent, er = ub.uncomp_entropy(ctx, K, k_trunc=k_trunc, center=center, norm=norm)
+    torch.cuda.synchronize()
+    parity.check_entropy(wl, K, ent, er, range(wl.units), k_trunc=k_trunc, center=center, norm=norm)
+
+
+def test_entropy_closed_forms_on_device():
+    # rank-1 keys -> H = 0; +-a e_i rows -> H = ln m   (Appendix, proof of the entropy bounds)
+    ub = _ub()
+    N, H = 256, 2
+    K = torch.zeros(1, 1, H, N, 128, device="cuda", dtype=torch.float32)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    u = torch.randn(N, 1, generator=g, device="cuda")
+    v = torch.randn(1, 128, generator=g, device="cuda")
+    K[0, 0, 0] = u @ v
+    m = 8
+    for i in range(m):
+        K[0, 0, 1, 2 * i, i] = 1.5
+        K[0, 0, 1, 2 * i + 1, i] = -1.5
+    ctx = ub.Context(ub.make_shape(1, 1, H, H, N, 128, 8, "fp32"))
+    ent, er = ub.uncomp_entropy(ctx, K, k_trunc=32)
+    torch.cuda.synchronize()
+    assert abs(float(ent[0, 0, 0])) < 1e-6 and abs(float(er[0, 0, 0]) - 1.0) < 1e-6
+    assert abs(float(ent[0, 0, 1]) - np.log(m)) < 1e-6 and abs(float(er[0, 0, 1]) - m) < 1e-5
+
+
+@pytest.mark.parametrize("scope,M,avg,n_max", [(0, 8, 100, 160), (1, 8, 100, 160), (0, 3, 77, 120), (1, 5, 64, 100),
+                                               (0, 1, 50, 50), (1, 24, 200, 360)])
+def test_budget_variants_bit_exact(scope, M, avg, n_max):
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=512, L=3, B=2)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    er = torch.rand(wl.B, wl.L, wl.H, generator=g, device="cuda") * 30 + 1
+    er[0, 1, 2] = er[0, 1, 5]
+    er[1, 0, 0] = er[1, 2, 7]
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    b, o, lg, lc = ub.uncomp_assign_budgets(ctx, er, avg, M, n_max, scope, eps=0.25, dn=64, n_last=128)
+    torch.cuda.synchronize()
+    parity.check_budgets(wl, er, b, o, lg, lc, M=M, avg=avg, n_max=n_max, scope=scope, eps=0.25, dn=64, n_last=128)
+    assert int(b.sum()) == wl.units * avg
+
+
+def test_budget_prefix_sum_beyond_one_block():
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=512, L=40, B=5)      # 1600 units > 1024 threads
+    g = torch.Generator(device="cuda").manual_seed(4)
+    er = torch.rand(wl.B, wl.L, wl.H, generator=g, device="cuda") * 30 + 1
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    b, o, lg, lc = ub.uncomp_assign_budgets(ctx, er, 100, 8, 160, 1)
+    torch.cuda.synchronize()
+    parity.check_budgets(wl, er, b, o, lg, lc, M=8, avg=100, n_max=160, scope=1)
+
+
+@pytest.mark.parametrize("w,G,N,pool,mode", [(1, 1, 300, 1, 0), (8, 4, 515, 7, 0), (32, 2, 1027, 5, 1),
+                                             (64, 8, 700, 7, 0), (17, 3, 401, 13, 1)])
+def test_scorer_shapes(w, G, N, pool, mode):
+    ub = _ub()
+    base = synth.scaled(synth.WORKLOADS["c2"], N=N, L=1)
+    from dataclasses import replace
+    wl = replace(base, w=w, Hq=base.H * G, avg_budget=w + 40, n_max=w + 40, M=1, pool_kernel=pool, pool_mode=mode)
+    K, V, Qw = synth.generate(wl, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    er = torch.ones(wl.B, wl.L, wl.H, device="cuda")
+    b, o, _, _ = ub.uncomp_assign_budgets(ctx, er, wl.avg_budget, 1, wl.n_max)
+    scores = torch.empty(wl.B, wl.L, wl.H, N - w, device="cuda")
+    idx = ub.uncomp_score_select(ctx, Qw, K, b, o, wl.total_rows, pool, mode, 0.0, scores)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    parity.check_scores(wl, K, Qw, scores, range(wl.units))
+    parity.check_select(wl, scores, b, o, idx, range(wl.units))
+    # mass conservation: probabilities of a row sum to one, so the prefix mass is at most G * w
+    if pool == 1:
+        assert float(scores.sum(-1).max()) <= G * w * (1 + 1e-4)
+
+
+@pytest.mark.parametrize("avg_kind", ["window_only", "one", "everything"])
+def test_select_extreme_budgets(avg_kind):
+    ub = _ub()
+    from dataclasses import replace
+    base = synth.scaled(synth.WORKLOADS["c2"], N=600, L=1)
+    avg = {"window_only": base.w, "one": base.w + 1, "everything": base.N}[avg_kind]
+    wl = replace(base, avg_budget=avg, n_max=avg, M=1)
+    K, V, Qw, cp, out = _run(wl)
+    parity.check_select(wl, out.scores, out.budgets, out.offsets, out.indices, range(wl.units))
+    parity.check_compact(wl, K, V, out.indices, out.offsets, out.Kc, out.Vc, range(wl.units))
+    if avg_kind == "everything":
+        assert torch.equal(out.Kc.view(wl.units, wl.N, wl.d), K.view(wl.units, wl.N, wl.d))
+
+
+def test_select_ties_take_lowest_positions():
+    # all keys equal -> every prefix score is equal -> the first k positions are kept
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=400, L=1)
+    K, V, Qw = synth.generate(wl, "cuda")
+    K[:] = K[:, :, :, :1, :]
+    from paper_2410_03090_b200.compress import CompressionPass
+    cp = CompressionPass(wl, "cuda")
+    out = cp.run(K, V, Qw)
+    torch.cuda.synchronize()
+    off = out.offsets.cpu().numpy()
+    bud = out.budgets.reshape(-1).cpu().numpy()
+    idx = out.indices.cpu().numpy()
+    for u in range(wl.units):
+        k = bud[u] - wl.w
+        seg = idx[off[u]:off[u + 1]]
+        assert seg.tolist() == list(range(k)) + list(range(wl.N - wl.w, wl.N))
+
+
+def test_strided_inputs_and_determinism():
+    # K / V as views of a larger [L, B, H, N, 2, d] buffer (interleaved K and V), two runs bit-identical
+    from paper_2410_03090_b200.compress import CompressionPass
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=640, L=2, B=2)
+    K0, V0, Qw = synth.generate(wl, "cuda")
+    big = torch.empty(wl.L, wl.B, wl.H, wl.N, 2, wl.d, dtype=K0.dtype, device="cuda")
+    big[..., 0, :] = K0.permute(1, 0, 2, 3, 4)
+    big[..., 1, :] = V0.permute(1, 0, 2, 3, 4)
+    K = big[..., 0, :].permute(1, 0, 2, 3, 4)
+    V = big[..., 1, :].permute(1, 0, 2, 3, 4)
+    assert not K.is_contiguous()
+    cp = CompressionPass(wl, "cuda")
+    out = cp.run(K, V, Qw)
+    torch.cuda.synchronize()
+    first = [t.clone() for t in (out.entropy, out.budgets, out.scores, out.indices, out.Kc, out.Vc)]
+    cp2 = CompressionPass(wl, "cuda")
+    ref = cp2.run(K0, V0, Qw)
+    out = cp.run(K, V, Qw)
+    torch.cuda.synchronize()
+    for a, b, c in zip(first, (out.entropy, out.budgets, out.scores, out.indices, out.Kc, out.Vc),
+                       (ref.entropy, ref.budgets, ref.scores, ref.indices, ref.Kc, ref.Vc)):
+        assert torch.equal(a, b) and torch.equal(a, c)
+    _check_all(wl, K0, V0, Qw, out, range(0, wl.units, 5))
+
+
+def test_host_side_rejections_and_status_word():
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=512, L=1)
+    K, V, Qw = synth.generate(wl, "cuda")
+    shape = ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype)
+    ctx = ub.Context(shape)
+    er = torch.ones(wl.B, wl.L, wl.H, device="cuda")
+
+    def code(fn, *a, **k):
+        with pytest.raises(ub.UncompError) as ei:
+            fn(*a, **k)
+        return ei.value.code
+
+    assert code(ub.uncomp_entropy, ctx, K, k_trunc=0) == ub.UNCOMP_E_PARAM
+    assert code(ub.uncomp_entropy, ctx, K.view(-1)[1:1 + 8 * 511 * 128].view(1, 1, 8, 511, 128)) == ub.UNCOMP_E_ALIGN
+    assert code(ub.uncomp_assign_budgets, ctx, er, 100, 9, 160) == ub.UNCOMP_E_PARAM       # M > heads
+    assert code(ub.uncomp_assign_budgets, ctx, er, 16, 8, 20) == ub.UNCOMP_E_PARAM         # avg < w
+    assert code(ub.uncomp_assign_budgets, ctx, er, 100, 8, 190) == ub.UNCOMP_E_PARAM       # smallest target < w
+    assert code(ub.uncomp_assign_budgets, ctx, er, 100, 8, 1000) == ub.UNCOMP_E_PARAM      # n_max > N
+    b, o, _, _ = ub.uncomp_assign_budgets(ctx, er, 100, 8, 160)
+    assert code(ub.uncomp_score_select, ctx, Qw, K, b, o, wl.units * 100, pool_kernel=4) == ub.UNCOMP_E_PARAM
+    # a workspace that is too small is refused at creation
+    import ctypes as C
+    h = C.c_void_p()
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    assert ub.lib.uncomp_create(C.byref(h), C.byref(shape), C.c_void_p(small.data_ptr()), 1024) == ub.UNCOMP_E_WORKSPACE
+    # device-side conditions arrive through the status word and leave the context usable
+    ub.uncomp_entropy(ctx, K, max_iters=1)
+    assert ub.uncomp_status(ctx) & ub.UNCOMP_STATUS_NOT_CONVERGED
+    bad = b.clone()
+    bad[0, 0, 0] = wl.N + 5
+    ub.uncomp_score_select(ctx, Qw, K, bad, o, wl.units * 100)
+    assert ub.uncomp_status(ctx) & ub.UNCOMP_STATUS_BOUNDS
+    ent, _ = ub.uncomp_entropy(ctx, K)
+    assert ub.uncomp_status(ctx) == 0
+    parity.check_entropy(wl, K, ent, _, [0, 5])
