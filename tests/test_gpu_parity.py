@@ -104,7 +104,7 @@ def test_entropy_closed_forms_on_device():
     assert abs(float(ent[0, 0, 1]) - np.log(m)) < 1e-6 and abs(float(er[0, 0, 1]) - m) < 1e-5
 
 
-@pytest.mark.parametrize("scope,M,avg,n_max", [(0, 8, 100, 160), (1, 8, 100, 160), (0, 3, 77, 120), (1, 5, 64, 100),
+@pytest.mark.parametrize("scope,M,avg,n_max", [(0, 8, 100, 160), (1, 8, 100, 160), (0, 3, 77, 120), (1, 5, 64, 96),
                                                (0, 1, 50, 50), (1, 24, 200, 360)])
 def test_budget_variants_bit_exact(scope, M, avg, n_max):
     ub = _ub()
