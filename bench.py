@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the UNComp prefill-end KV-compression pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl ours|reference]
+
+One step = one whole pass (entropy -> budgets -> window scores + selection -> compaction) over one batch
+of synthetic input.  Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own
+replica-sized shard (its own sequence of the same shape: units are independent, no collective on the
+data path) and the value is the sum over ranks divided by the slowest rank's time.
+
+`--impl reference` times the plain fp64 CPU oracle (oracle/) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from dataclasses import replace
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compression_pass_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_burst": float(p["bf16_tflops"]),
+                "bf16_sustained": float(p["bf16_tflops_sustained"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML (read-only) while the timed region runs."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, device_index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.power = [], set(), []
+        self.max_mhz = None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._halt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    bits = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def stop(self):
+        self._halt.set()
+        if self.is_alive():
+            self.join(timeout=2.0)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s), "power_w_max": round(max(self.power), 1) if self.power else None}
+
+
+# ------------------------------------------------------------------------------------- roofline per kernel
+def kernel_specs(wl, peaks, sustained: bool):
+    """Algorithmic work of one launch of each kernel of the pass (units of one rank)."""
+    u, N, d, P = wl.units, wl.N, wl.d, wl.N - wl.w
+    rows, s = wl.G * wl.w, wl.elem_bytes
+    tens = peaks["bf16_sustained"] if sustained else peaks["bf16_burst"]
+    if wl.dtype == "fp32":
+        tens = tens / 2.0 / 16.0   # fp32 inputs run on the CUDA cores; no tensor peak applies
+    hbm = peaks["hbm_gbs"]
+    return {
+        "gram": ("tensor", 2.0 * N * d * d * u / 1e12, tens, "TFLOP/s"),
+        "score_stats": ("tensor", 2.0 * rows * d * N * u / 1e12, tens, "TFLOP/s"),
+        "score_colsum": ("tensor", 2.0 * rows * d * P * u / 1e12, tens, "TFLOP/s"),
+        "pool_select": ("hbm", (2.0 * u * P * 4 + wl.total_rows * 4) / 1e9, hbm, "GB/s"),
+        "compact": ("hbm", wl.total_rows * (4.0 * d * s + 4) / 1e9, hbm, "GB/s"),
+        "eigen_entropy": ("alu", None, None, None),
+        "budgets": ("alu", None, None, None),
+        "stats_merge": ("hbm", None, None, None),
+    }
+
+
+# ------------------------------------------------------------------------------------------ oracle timing
+def time_oracle(wl, unit_list, fetch, threads, data=None):
+    """Wall time of the oracle chain over the given units, one thread per unit where possible.
+    The entropy and score stages (all the floating-point work) run in parallel over units; the budget
+    rule needs every head of a layer and runs once per layer."""
+    import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
+    import oracle
+    if data is None:
+        data = [fetch(u) for u in unit_list]
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        er = list(ex.map(lambda kvq: oracle.entropy(kvq[0], k_trunc=wl.k_trunc)[1], data))
+    n = len(data)
+    M = min(wl.M, n)
+    n_max = wl.n_max
+    bud, off, _, _ = oracle.budgets(np.array(er, dtype=np.float32).astype(np.float64).reshape(1, 1, n), wl.N, wl.w,
+                                    wl.avg_budget, M, n_max)
+
+    def rest(i):
+        K, V, Q = data[i]
+        sc = oracle.pool(oracle.window_scores(Q, K), wl.pool_kernel, wl.pool_mode)
+        idx = oracle.select(sc, wl.w, int(bud[0, 0, i]))
+        oracle.compact(np.ascontiguousarray(K).view(np.uint8).reshape(wl.N, -1), idx)
+        oracle.compact(np.ascontiguousarray(V).view(np.uint8).reshape(wl.N, -1), idx)
+        return len(idx)
+
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(rest, range(n)))
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    """The oracle as the reference arm: rank 0 only, CPU only, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from paper_2410_03090_b200 import synth
+    wl = synth.WORKLOADS[args.workload]
+    threads = min(os.cpu_count() or 1, 16)
+    total_steps = args.steps + args.warmup
+    per_step = wl.H if total_steps <= 30 else max(1, (30 * wl.H) // total_steps)
+    per_step = max(1, min(per_step, wl.H))
+
+    def fetch(u):
+        b, l, h = synth.unit_index(wl, u)
+        K, V, Q = synth.generate_unit(wl, b, l, h, "cpu", synth.spike_positions(wl, b))
+        return K.double().numpy(), V.double().numpy(), Q.double().numpy()
+
+    layer_units = list(range(per_step))
+    data = [fetch(u) for u in layer_units]
+    times = []
+    for s in range(total_steps):
+        t = time_oracle(wl, layer_units, fetch, threads, data)
+        if s >= args.warmup:
+            times.append(t)
+    t_step = sum(times) / len(times)
+    # tokens/s of the whole workload at this rate: the sample is per_step of wl.units units
+    value = wl.B * wl.N / (t_step * wl.units / per_step)
+    sample = f"{per_step} of {wl.units} units (heads 0..{per_step - 1} of layer 0) per step, whole oracle chain"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": _workload_name(wl), "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def _workload_name(wl):
+    return (f"{wl.name}: B{wl.B} L{wl.L} Hkv{wl.H} Hq{wl.Hq} N{wl.N} d{wl.d} w{wl.w} {wl.dtype}, "
+            f"avg budget {wl.avg_budget}, M{wl.M}, n_max {wl.n_max}, k{wl.k_trunc}")
+
+
+# ---------------------------------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c3")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2410_03090_b200 import binding as ub
+    from paper_2410_03090_b200 import synth
+    from paper_2410_03090_b200.compress import CompressionPass
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pass has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group(backend="nccl", device_id=dev)
+
+    base = synth.WORKLOADS[args.workload]
+    wl = replace(base, seed=base.seed + 7919 * rank)      # every rank compresses its own sequence(s)
+    peaks = _peaks()
+    K, V, Qw = synth.generate(wl, dev)
+    cp = CompressionPass(wl, dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    for _ in range(args.warmup):
+        cp.run(K, V, Qw)
+    torch.cuda.synchronize()
+    assert cp.status() == 0
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ub.uncomp_profile_enable(cp.ctx, True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        cp.run(K, V, Qw)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    prof = ub.uncomp_profile_read(cp.ctx)
+    ub.uncomp_profile_enable(cp.ctx, False)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    tokens_step = wl.B * wl.N * world
+    value = tokens_step / (ms_step / 1e3)
+
+    # ---- per-kernel roofline, from the events the library recorded inside the timed region
+    specs = kernel_specs(wl, peaks, sustained=True)
+    kernels = {}
+    launches = 0
+    for name, (ms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        launches += cnt
+        bound, work, peak, unit = specs[name]
+        avg_ms = ms / cnt
+        ent = {"launches_per_step": cnt // args.steps, "avg_ms": round(avg_ms, 5), "share": None, "bound": bound}
+        if work is not None:
+            ach = work / (avg_ms / 1e3)
+            ent.update({"achieved": round(ach, 2), "peak": peak, "unit": unit, "frac": round(ach / peak, 4)})
+        kernels[name] = ent
+    total_kernel_ms = sum(v[0] for v in prof.values())
+    for name in kernels:
+        kernels[name]["share"] = round(prof[name][0] / total_kernel_ms, 4)
+    dom = max(kernels, key=lambda n: kernels[n]["share"])
+    kd = kernels[dom]
+    roofline = {"kernel": dom, "bound": kd["bound"], "achieved": kd.get("achieved"), "peak": kd.get("peak"),
+                "unit": kd.get("unit"), "frac": kd.get("frac"), "traffic": None,
+                "peak_source": f"of {peaks['source']} ({'sustained bf16' if kd['bound'] == 'tensor' else 'copy'})",
+                "avg_ms": kd["avg_ms"], "share": kd["share"]}
+    alg_bytes = wl.algorithmic_bytes()
+    hbm_pass = alg_bytes / 1e9 / (ms_step / 1e3)
+
+    # ---- end to end: host buffers in, results out, copies inside the timed region
+    e2e = None
+    if args.e2e_steps > 0:
+        hK = torch.empty(K.shape, dtype=K.dtype, pin_memory=True).copy_(K)
+        hV = torch.empty(V.shape, dtype=V.dtype, pin_memory=True).copy_(V)
+        hQ = torch.empty(Qw.shape, dtype=Qw.dtype, pin_memory=True).copy_(Qw)
+        o = cp.out
+        outs = [o.Kc, o.Vc, o.indices, o.offsets, o.budgets, o.entropy]
+        houts = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+        dK, dV, dQ = torch.empty_like(K), torch.empty_like(V), torch.empty_like(Qw)
+        h2d = sum(t.numel() * t.element_size() for t in (hK, hV, hQ))
+        d2h = sum(t.numel() * t.element_size() for t in outs)
+
+        def e2e_step():
+            dK.copy_(hK, non_blocking=True)
+            dV.copy_(hV, non_blocking=True)
+            dQ.copy_(hQ, non_blocking=True)
+            cp.run(dK, dV, dQ)
+            for h, t in zip(houts, outs):
+                h.copy_(t, non_blocking=True)
+
+        e2e_step()
+        torch.cuda.synchronize()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+        ms_e = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms_e], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e = float(t.item())
+        e2e = {"value": tokens_step / (ms_e / args.e2e_steps / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+        del hK, hV, hQ, dK, dV, dQ
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, single GPU only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        threads = min(os.cpu_count() or 1, 16)
+        n_units = min(wl.units, 2 * wl.H)
+        layers = [0] if wl.L == 1 else [0, wl.L // 2]
+        unit_list = [l * wl.H + h for l in layers for h in range(wl.H)][:n_units]
+
+        def fetch(u):
+            b, l, h = synth.unit_index(wl, u)
+            return (K[b, l, h].double().cpu().numpy(), V[b, l, h].double().cpu().numpy(),
+                    Qw[b, l, h * wl.G:(h + 1) * wl.G].double().cpu().numpy())
+
+        t_cpu = 0.0
+        for l in layers:
+            ul = [x for x in unit_list if x // wl.H == l]
+            t_cpu += time_oracle(wl, ul, fetch, threads)
+        v = wl.B * wl.N / (t_cpu * wl.units / len(unit_list))
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
+                        "sample": f"{len(unit_list)} of {wl.units} units (all heads of layers {layers}), whole oracle "
+                                  f"chain, {t_cpu:.1f} s wall"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+                "config": {"workload": _workload_name(wl), "l2": "inputs larger than L2 (K+V = "
+                           f"{2 * K.numel() * K.element_size() / 1e9:.2f} GB streamed every step)",
+                           "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+                "hbm_pass": {"algorithmic_gb": round(alg_bytes / 1e9, 4), "achieved_gbs": round(hbm_pass, 1),
+                             "frac_of_measured_copy": round(hbm_pass / peaks["hbm_gbs"], 4),
+                             "frac_of_nominal_8tbs": round(hbm_pass / 8000.0, 4)},
+                "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
+                "gpu_launches": launches, "clocks": clocks}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

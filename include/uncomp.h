@@ -202,6 +202,18 @@ int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_str
  * that waits for the device. */
 int uncomp_status(uncomp_ctx *ctx, void *stream, uint32_t *host_bits);
 
+/* ---------------------------------------------------------------------------------------------------
+ * Per-kernel timing (no counterpart in the paper; it serves measurement).  While enabled, every kernel
+ * the four calls launch is bracketed by a pair of CUDA events on the caller's stream.
+ * uncomp_profile_read waits for the recorded events, adds the elapsed milliseconds and the launch
+ * counts per kernel slot into ms_sum / launches (host arrays of max_slots entries) and forgets the
+ * records.  Events are host-side driver objects; no device memory is allocated.
+ * ------------------------------------------------------------------------------------------------- */
+int uncomp_profile_enable(uncomp_ctx *ctx, int on);
+int uncomp_profile_slots(void);
+const char *uncomp_profile_slot_name(int slot);
+int uncomp_profile_read(uncomp_ctx *ctx, int max_slots, float *ms_sum, int32_t *launches);
+
 /* Text for a return code; never NULL. */
 const char *uncomp_strerror(int code);
 

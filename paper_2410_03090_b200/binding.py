@@ -68,6 +68,13 @@ def _load() -> C.CDLL:
                                         fp, i32p, vp]
     lib.uncomp_compact.restype = C.c_int
     lib.uncomp_compact.argtypes = [vp, vp, vp, uncomp_strides, uncomp_strides, i32p, i64p, vp, vp, vp]
+    lib.uncomp_profile_enable.restype = C.c_int
+    lib.uncomp_profile_enable.argtypes = [vp, C.c_int]
+    lib.uncomp_profile_slots.restype = C.c_int
+    lib.uncomp_profile_slot_name.restype = C.c_char_p
+    lib.uncomp_profile_slot_name.argtypes = [C.c_int]
+    lib.uncomp_profile_read.restype = C.c_int
+    lib.uncomp_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.uncomp_status.restype = C.c_int
     lib.uncomp_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
     return lib
@@ -204,3 +211,16 @@ def uncomp_status(ctx: Context, stream=None) -> int:
     bits = C.c_uint32(0)
     _check(lib.uncomp_status(ctx.handle, _stream(stream), C.byref(bits)), "uncomp_status")
     return int(bits.value)
+
+
+def uncomp_profile_enable(ctx: Context, on: bool) -> None:
+    _check(lib.uncomp_profile_enable(ctx.handle, int(on)), "uncomp_profile_enable")
+
+
+def uncomp_profile_read(ctx: Context) -> dict:
+    """{kernel name: (total ms, launches)} since the last read; waits for the recorded events."""
+    n = lib.uncomp_profile_slots()
+    ms = (C.c_float * n)()
+    cnt = (C.c_int32 * n)()
+    _check(lib.uncomp_profile_read(ctx.handle, n, ms, cnt), "uncomp_profile_read")
+    return {lib.uncomp_profile_slot_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}

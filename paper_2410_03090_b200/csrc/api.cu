@@ -2,6 +2,7 @@
 // kernel launches of the four calls.  No device memory is allocated here.
 #include <math.h>
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
@@ -59,6 +60,31 @@ Plan make_plan(const uncomp_shape &s) {
     return p;
 }
 
+// Per-kernel timing: one (start, stop) event pair per launch, appended while profiling is on.
+struct Profiler {
+    struct Rec { int slot; cudaEvent_t start, stop; };
+    std::vector<Rec> recs;     // records in use
+    std::vector<Rec> pool;     // event pairs created earlier, reused after a reset
+    static constexpr size_t kMaxRecs = 1 << 16;
+};
+
+void prof_begin(Profiler *p, int slot, cudaStream_t st) {
+    if (p->recs.size() >= Profiler::kMaxRecs) return;
+    Profiler::Rec r;
+    if (!p->pool.empty()) { r = p->pool.back(); p->pool.pop_back(); }
+    else {
+        if (cudaEventCreate(&r.start) != cudaSuccess) return;
+        if (cudaEventCreate(&r.stop) != cudaSuccess) { cudaEventDestroy(r.start); return; }
+    }
+    r.slot = slot;
+    cudaEventRecord(r.start, st);
+    p->recs.push_back(r);
+}
+
+void prof_end(Profiler *p, cudaStream_t st) {
+    if (!p->recs.empty()) cudaEventRecord(p->recs.back().stop, st);
+}
+
 }  // namespace uncomp
 
 using namespace uncomp;
@@ -68,6 +94,8 @@ struct uncomp_ctx {
     unsigned char *ws;
     int last_cuda;
     int device;
+    Profiler *prof;   // NULL unless profiling is on
+    Profiler prof_store;
 };
 
 static int cuda_fail(uncomp_ctx *ctx, cudaError_t e) {
@@ -123,6 +151,7 @@ int uncomp_create(uncomp_ctx **out, const uncomp_shape *shape, void *d_workspace
     ctx->ws = static_cast<unsigned char *>(d_workspace);
     ctx->last_cuda = 0;
     ctx->device = 0;
+    ctx->prof = nullptr;
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + p.off_status, 0, 256);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -134,7 +163,42 @@ int uncomp_create(uncomp_ctx **out, const uncomp_shape *shape, void *d_workspace
     return UNCOMP_OK;
 }
 
-void uncomp_destroy(uncomp_ctx *ctx) { delete ctx; }
+void uncomp_destroy(uncomp_ctx *ctx) {
+    if (!ctx) return;
+    for (auto &r : ctx->prof_store.recs) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+    for (auto &r : ctx->prof_store.pool) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+    delete ctx;
+}
+
+int uncomp_profile_enable(uncomp_ctx *ctx, int on) {
+    if (!ctx) return UNCOMP_E_NULL;
+    ctx->prof = on ? &ctx->prof_store : nullptr;
+    return UNCOMP_OK;
+}
+
+int uncomp_profile_slots(void) { return kSlotCount; }
+
+const char *uncomp_profile_slot_name(int slot) {
+    static const char *names[kSlotCount] = {"gram", "eigen_entropy", "budgets", "score_stats", "stats_merge",
+                                            "score_colsum", "pool_select", "compact"};
+    return slot >= 0 && slot < kSlotCount ? names[slot] : "";
+}
+
+int uncomp_profile_read(uncomp_ctx *ctx, int max_slots, float *ms_sum, int32_t *launches) {
+    if (!ctx || !ms_sum || !launches) return UNCOMP_E_NULL;
+    for (int i = 0; i < max_slots; ++i) { ms_sum[i] = 0.f; launches[i] = 0; }
+    Profiler &P = ctx->prof_store;
+    for (auto &r : P.recs) {
+        cudaError_t e = cudaEventSynchronize(r.stop);
+        float ms = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, r.start, r.stop);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        if (r.slot < max_slots) { ms_sum[r.slot] += ms; launches[r.slot] += 1; }
+        P.pool.push_back(r);
+    }
+    P.recs.clear();
+    return UNCOMP_OK;
+}
 
 int uncomp_last_cuda_error(const uncomp_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
 
@@ -152,9 +216,16 @@ int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const un
     uint32_t *d_status = reinterpret_cast<uint32_t *>(ctx->ws + p.off_status);
     void *partials = ctx->ws + p.off_gram;
     const UnitAddr addr = make_addr(p.shape, sK);
-    cudaError_t e = launch_gram_simt(p, d_K, addr, partials, st);
+    cudaError_t e;
+    {
+        ProfScope ps(ctx->prof, kSlotGram, st);
+        e = launch_gram_simt(p, d_K, addr, partials, st);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = launch_eigen_entropy(p, partials, *params, d_entropy, d_erank, d_spectrum, d_status, st);
+    {
+        ProfScope ps(ctx->prof, kSlotEigen, st);
+        e = launch_eigen_entropy(p, partials, *params, d_entropy, d_erank, d_spectrum, d_status, st);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;
 }
@@ -169,9 +240,13 @@ int uncomp_assign_budgets(uncomp_ctx *ctx, const float *d_erank, const uncomp_bu
     if (rc != UNCOMP_OK) return rc;
     if ((d_layer_group == nullptr) != (d_layer_ctx == nullptr)) return UNCOMP_E_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_budgets(p, d_erank, *params, d_budgets, d_offsets, d_layer_group, d_layer_ctx,
-                                   reinterpret_cast<int32_t *>(ctx->ws + p.off_rank),
-                                   reinterpret_cast<int64_t *>(ctx->ws + p.off_rem), st);
+    cudaError_t e;
+    {
+        ProfScope ps(ctx->prof, kSlotBudgets, st);
+        e = launch_budgets(p, d_erank, *params, d_budgets, d_offsets, d_layer_group, d_layer_ctx,
+                           reinterpret_cast<int32_t *>(ctx->ws + p.off_rank),
+                           reinterpret_cast<int64_t *>(ctx->ws + p.off_rem), st);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;
 }
@@ -195,10 +270,13 @@ int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, unco
     float *raw = reinterpret_cast<float *>(ctx->ws + p.off_raw);
     float *pooled = d_scores ? d_scores : reinterpret_cast<float *>(ctx->ws + p.off_pooled);
     const UnitAddr addr = make_addr(p.shape, sK);
-    cudaError_t e = launch_scores_simt(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, st);
+    cudaError_t e = launch_scores_simt(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, ctx->prof, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    e = launch_pool_select(p, raw, pooled, params->pool_kernel, params->pool_mode, d_budgets, d_offsets, d_indices,
-                           d_status, st);
+    {
+        ProfScope ps(ctx->prof, kSlotPoolSelect, st);
+        e = launch_pool_select(p, raw, pooled, params->pool_kernel, params->pool_mode, d_budgets, d_offsets,
+                               d_indices, d_status, st);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;
 }
@@ -213,8 +291,12 @@ int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_str
     rc = check_strides(p.shape, sV);
     if (rc != UNCOMP_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_compact(p, d_K, d_V, make_addr(p.shape, sK), make_addr(p.shape, sV), d_indices,
-                                   d_offsets, d_Kc, d_Vc, st);
+    cudaError_t e;
+    {
+        ProfScope ps(ctx->prof, kSlotCompact, st);
+        e = launch_compact(p, d_K, d_V, make_addr(p.shape, sK), make_addr(p.shape, sV), d_indices, d_offsets, d_Kc,
+                           d_Vc, st);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;
 }

@@ -58,6 +58,18 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
+// Optional per-kernel timing with CUDA events on the launching stream (host objects only).
+enum Slot { kSlotGram = 0, kSlotEigen, kSlotBudgets, kSlotScoreStats, kSlotStatsMerge, kSlotScoreColsum,
+            kSlotPoolSelect, kSlotCompact, kSlotCount };
+struct Profiler;
+void prof_begin(Profiler *p, int slot, cudaStream_t st);
+void prof_end(Profiler *p, cudaStream_t st);
+struct ProfScope {
+    Profiler *p; cudaStream_t st;
+    ProfScope(Profiler *p_, int slot, cudaStream_t st_) : p(p_), st(st_) { if (p) prof_begin(p, slot, st); }
+    ~ProfScope() { if (p) prof_end(p, st); }
+};
+
 // ---- kernel launchers (each returns the cudaError_t of its launches) -------------------------------
 cudaError_t launch_gram_simt(const Plan &p, const void *dK, const UnitAddr &addr, void *d_partials, cudaStream_t st);
 cudaError_t launch_eigen_entropy(const Plan &p, const void *d_partials, const uncomp_entropy_params &ep,
@@ -68,7 +80,7 @@ cudaError_t launch_budgets(const Plan &p, const float *d_erank, const uncomp_bud
                            int64_t *d_offsets, int32_t *d_layer_group, int32_t *d_layer_ctx, int32_t *d_rank,
                            int64_t *d_rem, cudaStream_t st);
 cudaError_t launch_scores_simt(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
-                               float *d_stats_part, float *d_stats, float *d_raw, cudaStream_t st);
+                               float *d_stats_part, float *d_stats, float *d_raw, Profiler *prof, cudaStream_t st);
 cudaError_t launch_pool_select(const Plan &p, const float *d_raw, float *d_pooled, int pool_kernel, int pool_mode,
                                const int32_t *d_budgets, const int64_t *d_offsets, int32_t *d_indices,
                                uint32_t *d_status, cudaStream_t st);

@@ -173,7 +173,8 @@ __global__ void __launch_bounds__(256) score_colsum_simt_kernel(const T *__restr
 
 template <typename T>
 static cudaError_t launch_scores_simt_t(const Plan &p, const T *dQw, const T *dK, const UnitAddr &addr, float scale,
-                                        float *d_stats_part, float *d_stats, float *d_raw, cudaStream_t st) {
+                                        float *d_stats_part, float *d_stats, float *d_raw, Profiler *prof,
+                                        cudaStream_t st) {
     const size_t smemA = 2 * kSB * kKPad * sizeof(float);
     const size_t smemB = smemA + 16 * kSB * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(score_stats_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -183,24 +184,33 @@ static cudaError_t launch_scores_simt_t(const Plan &p, const T *dQw, const T *dK
     if (e != cudaSuccess) return e;
     const int row_blocks = (p.rows + kSB - 1) / kSB;
     dim3 gA(p.score_splits, row_blocks, p.units);
-    score_stats_simt_kernel<T><<<gA, 256, smemA, st>>>(dQw, dK, addr, p.shape.N, p.shape.w, p.G, p.score_chunk,
-                                                       p.score_splits, scale, d_stats_part);
+    {
+        ProfScope ps(prof, kSlotScoreStats, st);
+        score_stats_simt_kernel<T><<<gA, 256, smemA, st>>>(dQw, dK, addr, p.shape.N, p.shape.w, p.G, p.score_chunk,
+                                                           p.score_splits, scale, d_stats_part);
+    }
     const int total = p.units * p.rows;
-    score_stats_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows, p.score_splits,
-                                                                  d_stats);
+    {
+        ProfScope ps(prof, kSlotStatsMerge, st);
+        score_stats_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows, p.score_splits,
+                                                                      d_stats);
+    }
     dim3 gB((p.prefix + kSB - 1) / kSB, p.units);
-    score_colsum_simt_kernel<T><<<gB, 256, smemB, st>>>(dQw, dK, addr, p.shape.N, p.shape.w, p.G, scale, d_stats,
-                                                        d_raw);
+    {
+        ProfScope ps(prof, kSlotScoreColsum, st);
+        score_colsum_simt_kernel<T><<<gB, 256, smemB, st>>>(dQw, dK, addr, p.shape.N, p.shape.w, p.G, scale, d_stats,
+                                                            d_raw);
+    }
     return cudaGetLastError();
 }
 
 cudaError_t launch_scores_simt(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
-                               float *d_stats_part, float *d_stats, float *d_raw, cudaStream_t st) {
+                               float *d_stats_part, float *d_stats, float *d_raw, Profiler *prof, cudaStream_t st) {
     if (p.shape.dtype == UNCOMP_FP32)
         return launch_scores_simt_t<float>(p, (const float *)dQw, (const float *)dK, addr, scale, d_stats_part,
-                                           d_stats, d_raw, st);
+                                           d_stats, d_raw, prof, st);
     return launch_scores_simt_t<__nv_bfloat16>(p, (const __nv_bfloat16 *)dQw, (const __nv_bfloat16 *)dK, addr, scale,
-                                               d_stats_part, d_stats, d_raw, st);
+                                               d_stats_part, d_stats, d_raw, prof, st);
 }
 
 }  // namespace uncomp
