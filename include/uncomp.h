@@ -114,6 +114,12 @@ typedef struct {
 int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const uncomp_entropy_params *params,
                    float *d_entropy, float *d_erank, double *d_spectrum, void *stream);
 
+/* uncomp_gram -- the building blocks of Eq. 1 on their own: for every unit the Gram matrix G = X^T X and
+ * the column sums s = X^T 1 (the covariance of Eq. 1 is (G - s s^T / N) / (N - 1)), as produced by the
+ * first stage of uncomp_entropy and summed over its token chunks in fp64.
+ * d_gram  out  [B*L*H, d*d + d] double: G row-major, then s. */
+int uncomp_gram(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, double *d_gram, void *stream);
+
 /* ---------------------------------------------------------------------------------------------------
  * uncomp_assign_budgets -- Section 3.3.3 "Head-Group Compression": heads ranked by truncated effective
  * rank, split into M groups, group budgets N_{i,g+1} = N_{i,g} - step from n_max downwards; and
@@ -201,6 +207,12 @@ int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_str
 /* Synchronise `stream`, copy the status word to *host_bits and clear it on the device.  The only call
  * that waits for the device. */
 int uncomp_status(uncomp_ctx *ctx, void *stream, uint32_t *host_bits);
+
+/* Options of a context (no counterpart in the paper).  UNCOMP_OPT_CUDA_CORES = 1 makes bf16 inputs take
+ * the plain CUDA-core kernels that fp32 inputs always use instead of the tensor-core kernels: a
+ * debugging aid for comparing the two. */
+enum { UNCOMP_OPT_CUDA_CORES = 1 };
+int uncomp_set_option(uncomp_ctx *ctx, int option, int value);
 
 /* ---------------------------------------------------------------------------------------------------
  * Per-kernel timing (no counterpart in the paper; it serves measurement).  While enabled, every kernel

@@ -61,6 +61,8 @@ def _load() -> C.CDLL:
     lib.uncomp_last_cuda_error.argtypes = [vp]
     lib.uncomp_entropy.restype = C.c_int
     lib.uncomp_entropy.argtypes = [vp, vp, uncomp_strides, C.POINTER(uncomp_entropy_params), fp, fp, dp, vp]
+    lib.uncomp_gram.restype = C.c_int
+    lib.uncomp_gram.argtypes = [vp, vp, uncomp_strides, dp, vp]
     lib.uncomp_assign_budgets.restype = C.c_int
     lib.uncomp_assign_budgets.argtypes = [vp, fp, C.POINTER(uncomp_budget_params), i32p, i64p, i32p, i32p, vp]
     lib.uncomp_score_select.restype = C.c_int
@@ -68,6 +70,8 @@ def _load() -> C.CDLL:
                                         fp, i32p, vp]
     lib.uncomp_compact.restype = C.c_int
     lib.uncomp_compact.argtypes = [vp, vp, vp, uncomp_strides, uncomp_strides, i32p, i64p, vp, vp, vp]
+    lib.uncomp_set_option.restype = C.c_int
+    lib.uncomp_set_option.argtypes = [vp, C.c_int, C.c_int]
     lib.uncomp_profile_enable.restype = C.c_int
     lib.uncomp_profile_enable.argtypes = [vp, C.c_int]
     lib.uncomp_profile_slots.restype = C.c_int
@@ -163,6 +167,14 @@ def uncomp_entropy(ctx: Context, K: torch.Tensor, k_trunc: int = 32, center: int
     return entropy, erank
 
 
+def uncomp_gram(ctx: Context, K: torch.Tensor, gram: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    s = ctx.shape
+    if gram is None:
+        gram = torch.empty(s.B * s.L * s.H, s.d * s.d + s.d, dtype=torch.float64, device=K.device)
+    _check(lib.uncomp_gram(ctx.handle, _ptr(K), strides_of(K), _ptr(gram), _stream(stream)), "uncomp_gram")
+    return gram
+
+
 def uncomp_assign_budgets(ctx: Context, erank: torch.Tensor, avg_budget: int, M: int, n_max: int, scope: int = 0,
                           eps: float = 0.0, dn: int = 0, n_last: int = 0, budgets=None, offsets=None,
                           layer_group=None, layer_ctx=None, stream=None):
@@ -211,6 +223,13 @@ def uncomp_status(ctx: Context, stream=None) -> int:
     bits = C.c_uint32(0)
     _check(lib.uncomp_status(ctx.handle, _stream(stream), C.byref(bits)), "uncomp_status")
     return int(bits.value)
+
+
+UNCOMP_OPT_CUDA_CORES = 1
+
+
+def uncomp_set_option(ctx: Context, option: int, value: int) -> None:
+    _check(lib.uncomp_set_option(ctx.handle, option, value), "uncomp_set_option")
 
 
 def uncomp_profile_enable(ctx: Context, on: bool) -> None:

@@ -96,6 +96,7 @@ struct uncomp_ctx {
     int device;
     Profiler *prof;   // NULL unless profiling is on
     Profiler prof_store;
+    int force_simt;   // UNCOMP_OPT_CUDA_CORES
 };
 
 static int cuda_fail(uncomp_ctx *ctx, cudaError_t e) {
@@ -152,6 +153,7 @@ int uncomp_create(uncomp_ctx **out, const uncomp_shape *shape, void *d_workspace
     ctx->last_cuda = 0;
     ctx->device = 0;
     ctx->prof = nullptr;
+    ctx->force_simt = 0;
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + p.off_status, 0, 256);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -168,6 +170,12 @@ void uncomp_destroy(uncomp_ctx *ctx) {
     for (auto &r : ctx->prof_store.recs) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
     for (auto &r : ctx->prof_store.pool) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
     delete ctx;
+}
+
+int uncomp_set_option(uncomp_ctx *ctx, int option, int value) {
+    if (!ctx) return UNCOMP_E_NULL;
+    if (option == UNCOMP_OPT_CUDA_CORES) { ctx->force_simt = value != 0; return UNCOMP_OK; }
+    return UNCOMP_E_PARAM;
 }
 
 int uncomp_profile_enable(uncomp_ctx *ctx, int on) {
@@ -219,13 +227,33 @@ int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const un
     cudaError_t e;
     {
         ProfScope ps(ctx->prof, kSlotGram, st);
-        e = launch_gram_simt(p, d_K, addr, partials, st);
+        if (p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt) e = launch_gram_tc(p, d_K, addr, partials, d_status, st);
+        else e = launch_gram_simt(p, d_K, addr, partials, st);
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     {
         ProfScope ps(ctx->prof, kSlotEigen, st);
         e = launch_eigen_entropy(p, partials, *params, d_entropy, d_erank, d_spectrum, d_status, st);
     }
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+int uncomp_gram(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, double *d_gram, void *stream) {
+    if (!ctx || !d_K || !d_gram) return UNCOMP_E_NULL;
+    const Plan &p = ctx->plan;
+    if (!aligned16(d_K)) return UNCOMP_E_ALIGN;
+    int rc = check_strides(p.shape, sK);
+    if (rc != UNCOMP_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t *d_status = reinterpret_cast<uint32_t *>(ctx->ws + p.off_status);
+    void *partials = ctx->ws + p.off_gram;
+    const UnitAddr addr = make_addr(p.shape, sK);
+    cudaError_t e;
+    if (p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt) e = launch_gram_tc(p, d_K, addr, partials, d_status, st);
+    else e = launch_gram_simt(p, d_K, addr, partials, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    e = launch_gram_reduce(p, partials, d_gram, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;
 }

@@ -72,9 +72,12 @@ struct ProfScope {
 
 // ---- kernel launchers (each returns the cudaError_t of its launches) -------------------------------
 cudaError_t launch_gram_simt(const Plan &p, const void *dK, const UnitAddr &addr, void *d_partials, cudaStream_t st);
+cudaError_t launch_gram_tc(const Plan &p, const void *dK, const UnitAddr &addr, void *d_partials, uint32_t *d_status,
+                           cudaStream_t st);
 cudaError_t launch_eigen_entropy(const Plan &p, const void *d_partials, const uncomp_entropy_params &ep,
                                  float *d_entropy, float *d_erank, double *d_spectrum, uint32_t *d_status,
                                  cudaStream_t st);
+cudaError_t launch_gram_reduce(const Plan &p, const void *d_partials, double *d_out, cudaStream_t st);
 int check_budget_params(const uncomp_shape &s, const uncomp_budget_params &bp);
 cudaError_t launch_budgets(const Plan &p, const float *d_erank, const uncomp_budget_params &bp, int32_t *d_budgets,
                            int64_t *d_offsets, int32_t *d_layer_group, int32_t *d_layer_ctx, int32_t *d_rank,

@@ -238,6 +238,27 @@ eigen_entropy_kernel(const PartialT *__restrict__ partials, int P, int N, int k_
     if (spectrum && tid < k) spectrum[(size_t)u * k + tid] = S.lam[tid];
 }
 
+// Sum of the chunk partials of every unit in chunk order: out[u] = [G (d*d) | s (d)] in fp64.
+template <typename PartialT>
+__global__ void gram_reduce_kernel(const PartialT *__restrict__ partials, int P, double *__restrict__ out) {
+    constexpr int len = kD * kD + kD;
+    const int u = blockIdx.y;
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= len) return;
+    double g = 0.0;
+    for (int p = 0; p < P; ++p) g += (double)partials[((size_t)u * P + p) * len + e];
+    out[(size_t)u * len + e] = g;
+}
+
+cudaError_t launch_gram_reduce(const Plan &p, const void *d_partials, double *d_out, cudaStream_t st) {
+    dim3 grid((kD * kD + kD + 255) / 256, p.units);
+    if (p.shape.dtype == UNCOMP_FP32)
+        gram_reduce_kernel<double><<<grid, 256, 0, st>>>((const double *)d_partials, p.gram_splits, d_out);
+    else
+        gram_reduce_kernel<float><<<grid, 256, 0, st>>>((const float *)d_partials, p.gram_splits, d_out);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_eigen_entropy(const Plan &p, const void *d_partials, const uncomp_entropy_params &ep,
                                  float *d_entropy, float *d_erank, double *d_spectrum, uint32_t *d_status,
                                  cudaStream_t st) {

@@ -247,3 +247,48 @@ def test_host_side_rejections_and_status_word():
     ent, _ = ub.uncomp_entropy(ctx, K)
     assert ub.uncomp_status(ctx) == 0
     parity.check_entropy(wl, K, ent, _, [0, 5])
+
+
+def _gram_oracle(K_unit_np):
+    import oracle
+    G = oracle.covariance(K_unit_np, center=False)
+    return G, K_unit_np.sum(axis=0)
+
+
+@pytest.mark.parametrize("N", [128, 200, 1000, 4096 + 77])
+def test_gram_known_answer_integers(N):
+    # integer-valued bf16 keys: every product and partial sum is exact in fp32, so the tensor-core Gram
+    # must equal the oracle's X^T X and column sums exactly (this pins operand layout, swizzle and tiling)
+    ub = _ub()
+    H = 3
+    g = torch.Generator(device="cuda").manual_seed(N)
+    K = torch.randint(-3, 4, (1, 1, H, N, 128), generator=g, device="cuda").to(torch.bfloat16)
+    K[0, 0, 1, :, 5] = 1.0          # a constant feature: its column sum is N
+    K[0, 0, 2, N - 1, :] = 7.0      # the last token must be counted once
+    ctx = ub.Context(ub.make_shape(1, 1, H, H, N, 128, 8, "bf16"))
+    gram = ub.uncomp_gram(ctx, K)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    for u in range(H):
+        G, s = _gram_oracle(K[0, 0, u].double().cpu().numpy())
+        got = gram[u].cpu().numpy()
+        np.testing.assert_array_equal(got[:128 * 128].reshape(128, 128), G)
+        np.testing.assert_array_equal(got[128 * 128:], s)
+
+
+def test_gram_tensor_core_vs_cuda_core_and_oracle():
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c3"], N=5000, L=2)
+    K, _, _ = synth.generate(wl, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    g_tc = ub.uncomp_gram(ctx, K).clone()
+    ub.uncomp_set_option(ctx, ub.UNCOMP_OPT_CUDA_CORES, 1)
+    g_cc = ub.uncomp_gram(ctx, K).clone()
+    torch.cuda.synchronize()
+    scale = g_cc[:, :128 * 128].abs().amax(dim=1, keepdim=True)
+    assert float(((g_tc - g_cc).abs() / scale).max()) < 2e-6
+    for u in (0, 9):
+        G, s = _gram_oracle(parity.unit_np(K, wl, u))
+        got = g_tc[u].cpu().numpy()
+        assert np.abs(got[:128 * 128].reshape(128, 128) - G).max() <= 2e-6 * np.abs(G).max()
+        assert np.abs(got[128 * 128:] - s).max() <= 2e-6 * np.abs(np.diag(G)).max() ** 0.5 * wl.N ** 0.5 + 1e-3
