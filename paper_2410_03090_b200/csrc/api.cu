@@ -39,10 +39,9 @@ Plan make_plan(const uncomp_shape &s) {
         p.gram_splits = (s.N + chunk - 1) / chunk;
     }
     {
-        int want = (target_ctas + p.units - 1) / p.units;
-        int most = (s.N + 511) / 512;
-        int P = want < 1 ? 1 : (want > most ? most : want);
-        int chunk = (int)align_up((size_t)(s.N + P - 1) / P, 64);
+        // scorer: chunks of 4096 tokens (a multiple of the 128-token tile), halved while the grid is small
+        int chunk = 4096;
+        while (chunk > 512 && (int64_t)p.units * ((s.N + chunk - 1) / chunk) < target_ctas) chunk >>= 1;
         p.score_chunk = chunk;
         p.score_splits = (s.N + chunk - 1) / chunk;
     }
@@ -50,7 +49,7 @@ Plan make_plan(const uncomp_shape &s) {
     size_t o = 0;
     p.off_status = o;      o = align_up(o + 256, 256);
     p.off_gram = o;        o = align_up(o + (size_t)p.units * p.gram_splits * (kD * kD + kD) * acc, 256);
-    p.off_stats_part = o;  o = align_up(o + (size_t)p.units * p.score_splits * kMaxRows * 2 * sizeof(float), 256);
+    p.off_stats_part = o;  o = align_up(o + (size_t)p.units * p.score_splits * 2 * kMaxRows * 2 * sizeof(float), 256);
     p.off_stats = o;       o = align_up(o + (size_t)p.units * kMaxRows * 2 * sizeof(float), 256);
     p.off_raw = o;         o = align_up(o + (size_t)p.units * p.prefix * sizeof(float), 256);
     p.off_pooled = o;      o = align_up(o + (size_t)p.units * p.prefix * sizeof(float), 256);
@@ -298,7 +297,11 @@ int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, unco
     float *raw = reinterpret_cast<float *>(ctx->ws + p.off_raw);
     float *pooled = d_scores ? d_scores : reinterpret_cast<float *>(ctx->ws + p.off_pooled);
     const UnitAddr addr = make_addr(p.shape, sK);
-    cudaError_t e = launch_scores_simt(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, ctx->prof, st);
+    cudaError_t e;
+    if (p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt)
+        e = launch_scores_tc(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, d_status, ctx->prof, st);
+    else
+        e = launch_scores_simt(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, ctx->prof, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     {
         ProfScope ps(ctx->prof, kSlotPoolSelect, st);

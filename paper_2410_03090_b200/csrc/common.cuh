@@ -84,6 +84,9 @@ cudaError_t launch_budgets(const Plan &p, const float *d_erank, const uncomp_bud
                            int64_t *d_rem, cudaStream_t st);
 cudaError_t launch_scores_simt(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
                                float *d_stats_part, float *d_stats, float *d_raw, Profiler *prof, cudaStream_t st);
+cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
+                             float *d_stats_part, float *d_stats, float *d_raw, uint32_t *d_status, Profiler *prof,
+                             cudaStream_t st);
 cudaError_t launch_pool_select(const Plan &p, const float *d_raw, float *d_pooled, int pool_kernel, int pool_mode,
                                const int32_t *d_budgets, const int64_t *d_offsets, int32_t *d_indices,
                                uint32_t *d_status, cudaStream_t st);

@@ -157,14 +157,7 @@ cudaError_t launch_gram_tc(const Plan &p, const void *dK, const UnitAddr &addr, 
                            cudaStream_t st) {
     const uncomp_shape &s = p.shape;
     CUtensorMap tmap;
-    // dims (feature, token, head, layer, batch); a dimension of extent 1 gets a harmless valid stride
-    uint64_t dims[5] = {(uint64_t)s.d, (uint64_t)s.N, (uint64_t)s.H, (uint64_t)s.L, (uint64_t)s.B};
-    uint64_t str[4] = {(uint64_t)addr.sN * 2, (uint64_t)addr.sH * 2, (uint64_t)addr.sL * 2, (uint64_t)addr.sB * 2};
-    for (int i = 0; i < 4; ++i)
-        if (dims[i + 1] == 1 && str[i] == 0) str[i] = (i == 0 ? (uint64_t)s.d * 2 : str[i - 1] * dims[i]);
-    uint32_t box[5] = {64, (uint32_t)kTile, 1, 1, 1};
-    cudaError_t e = encode_tensor_map(&tmap, dK, 5, dims, str, box, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-                                      CU_TENSOR_MAP_SWIZZLE_128B);
+    cudaError_t e = make_key_tensor_map(&tmap, s, addr, dK, kTile);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGramSmem);
     if (e != cudaSuccess) return e;

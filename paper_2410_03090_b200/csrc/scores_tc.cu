@@ -1,0 +1,327 @@
+// Observation-window scores for bf16 keys on the tcgen05 tensor cores (paper Section 3.3.3, "Dynamic KV
+// Cache Eviction": the attention of the last w query positions, summed per key position).
+//
+// Two kernels with one pipeline skeleton; softmax needs the row statistics before the column sums:
+//   pass A  S = Qw K^T with the window rows on the TMEM lanes (M = 128 rows, N = 128 tokens per MMA tile):
+//           a thread owns a row, so its running maximum and sum of exponentials are thread-local;
+//           every (unit, chunk, column half) writes partial statistics (m, l) in the log2 domain;
+//   merge   partials combined in index order into m'_r = m_r + log2 l_r;
+//   pass B  operands swapped (M = 128 tokens on the lanes, N = 128 rows): a thread owns a token and adds
+//           2^(s c - m'_r) along its TMEM row; tokens of a warp are consecutive, the store is coalesced.
+// K tiles (128 tokens x 128 features, two 128B-swizzled boxes of 64 features) stream through a TMA ring;
+// the unit's window queries stay in shared memory for the whole CTA.  Both operands are K-major.
+//
+// CTA = 320 threads on one SM: warps 0-7 softmax (warp % 4 selects the TMEM lane quarter, warp / 4 the
+// column half of an accumulator), warp 8 TMA producer, warp 9 TMEM allocation and MMA issue.  Four
+// 128-column accumulators rotate, so the tensor pipe runs ahead of the exponentials.
+// Every wait is bounded; a timeout raises UNCOMP_STATUS_TIMEOUT and the CTA drains and exits.
+#include "tc_common.cuh"
+
+namespace uncomp {
+
+namespace {
+constexpr int kTile = 128;
+constexpr int kHalfBytes = 128 * 128;            // 64 features x 128 rows/tokens, bf16
+constexpr int kBlockBytes = 2 * kHalfBytes;      // one K tile or one block of 128 query rows
+constexpr int kNB = 4;                           // accumulator buffers (x 128 TMEM columns = all 512)
+constexpr int kSoftThreads = 256;
+constexpr int kScoreThreads = kSoftThreads + 64;
+constexpr int kMaxStages = 4;
+
+struct ScoreTail {
+    uint64_t full[kMaxStages], empty[kMaxStages], qfull, tfull[kNB], tempty[kNB];
+    uint32_t tmem_base;
+};
+
+__host__ __device__ constexpr int score_stages(int MB) { return MB <= 2 ? 4 : (MB == 3 ? 3 : 2); }
+__host__ __device__ constexpr int score_smem(int MB) {
+    return 1024 + MB * kBlockBytes + score_stages(MB) * kBlockBytes + MB * 128 * 4 + 2 * 2 * 128 * 4 +
+           (int)sizeof(ScoreTail);
+}
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void soft_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+}  // namespace
+
+template <int MB, bool PASS_B>
+__global__ void __launch_bounds__(kScoreThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant__ CUtensorMap tmapK, int L, int H,
+                int N, int w, int rows, int chunk, int splits, float c_log2, float *__restrict__ stats_part,
+                const float *__restrict__ mprime, float *__restrict__ raw, uint32_t *__restrict__ status) {
+    constexpr int S = score_stages(MB);
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw_addr = tc::smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    unsigned char *smem = smem_raw + pad;
+    const uint32_t q_addr = raw_addr + pad;
+    const uint32_t k_addr = q_addr + MB * kBlockBytes;
+    float *mp = reinterpret_cast<float *>(smem + (MB + S) * kBlockBytes);      // [MB * 128]
+    float *colsum = mp + MB * 128;                                             // [2][2][128]
+    ScoreTail &T = *reinterpret_cast<ScoreTail *>(colsum + 2 * 2 * 128);
+
+    const int c = blockIdx.x, u = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = u % H, l = (u / H) % L, b = u / (H * L);
+    const int P = N - w;
+    const int limit = PASS_B ? P : N;              // pass B only scores the prefix
+    const int t0 = c * chunk;
+    const int t1 = min(limit, t0 + chunk);
+    const int ntiles = t1 > t0 ? (t1 - t0 + kTile - 1) / kTile : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            tc::mbar_init(tc::smem_u32(&T.full[s]), 1);
+            tc::mbar_init(tc::smem_u32(&T.empty[s]), 1);
+        }
+        tc::mbar_init(tc::smem_u32(&T.qfull), 1);
+        for (int i = 0; i < kNB; ++i) {
+            tc::mbar_init(tc::smem_u32(&T.tfull[i]), 1);
+            tc::mbar_init(tc::smem_u32(&T.tempty[i]), kSoftThreads / 32);
+        }
+        tc::fence_mbar_init();
+    }
+    if (warp == 9) {
+        tc::tmem_alloc(tc::smem_u32(&T.tmem_base), 512);
+        tc::tmem_relinquish();
+    }
+    if (warp == 8 && lane == 0) {
+        tc::prefetch_tmap(&tmapQ);
+        tc::prefetch_tmap(&tmapK);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem = T.tmem_base;
+
+    if (warp == 8) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0 && ntiles > 0) {
+            const uint32_t qbar = tc::smem_u32(&T.qfull);
+            tc::mbar_expect_tx(qbar, MB * kBlockBytes);
+            for (int mb = 0; mb < MB; ++mb) {
+                tc::tma_load_3d(q_addr + mb * kBlockBytes, &tmapQ, qbar, 0, mb * 128, u);
+                tc::tma_load_3d(q_addr + mb * kBlockBytes + kHalfBytes, &tmapQ, qbar, 64, mb * 128, u);
+            }
+            int issued = 0;
+            bool ok = true;
+            for (int i = 0; i < ntiles; ++i, ++issued) {
+                const int s = i % S;
+                if (i >= S) ok = tc::mbar_wait(tc::smem_u32(&T.empty[s]), ((i / S) - 1) & 1, status);
+                if (!ok) break;
+                const uint32_t bar = tc::smem_u32(&T.full[s]);
+                const uint32_t dst = k_addr + s * kBlockBytes;
+                tc::mbar_expect_tx(bar, kBlockBytes);
+                tc::tma_load_5d(dst, &tmapK, bar, 0, t0 + i * kTile, h, l, b);
+                tc::tma_load_5d(dst + kHalfBytes, &tmapK, bar, 64, t0 + i * kTile, h, l, b);
+            }
+            if (!ok) {   // let the copies in flight land before the CTA may exit (bounded)
+                tc::mbar_wait(qbar, 0, status);
+                for (int i = max(0, issued - S); i < issued; ++i)
+                    tc::mbar_wait(tc::smem_u32(&T.full[i % S]), (i / S) & 1, status);
+            }
+        }
+    } else if (warp == 9) {
+        // ---------------- MMA issue ----------------
+        if (lane == 0 && ntiles > 0) {
+            constexpr uint32_t idesc = tc::idesc_bf16_f32(128, 128, 0, 0);
+            bool ok = tc::mbar_wait(tc::smem_u32(&T.qfull), 0, status);
+            for (int i = 0; i < ntiles && ok; ++i) {
+                const int s = i % S;
+                ok = tc::mbar_wait(tc::smem_u32(&T.full[s]), (i / S) & 1, status);
+                if (!ok) break;
+                const uint32_t kbase = k_addr + s * kBlockBytes;
+                for (int mb = 0; mb < MB && ok; ++mb) {
+                    const int q = i * MB + mb, buf = q % kNB;
+                    if (q >= kNB) ok = tc::mbar_wait(tc::smem_u32(&T.tempty[buf]), ((q / kNB) - 1) & 1, status);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    const uint32_t qbase = q_addr + mb * kBlockBytes;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        // 16 features further = 32 B inside the 128-byte swizzle row; second half one region on
+                        const uint32_t off = (uint32_t)(k >> 2) * kHalfBytes + (uint32_t)(k & 3) * 32;
+                        const uint64_t qd = tc::smem_desc_sw128(qbase + off, 16, 1024);
+                        const uint64_t kd = tc::smem_desc_sw128(kbase + off, 16, 1024);
+                        if (PASS_B) tc::mma_f16_ss(tmem + buf * 128, kd, qd, idesc, k > 0);
+                        else tc::mma_f16_ss(tmem + buf * 128, qd, kd, idesc, k > 0);
+                    }
+                    tc::mma_commit(tc::smem_u32(&T.tfull[buf]));
+                }
+                tc::mma_commit(tc::smem_u32(&T.empty[s]));
+            }
+        }
+    } else {
+        // ---------------- softmax warps ----------------
+        const int quarter = warp & 3, hf = warp >> 2;
+        const int lane_row = quarter * 32 + lane;          // TMEM lane: a window row (A) or a token (B)
+        const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)hf * 64;
+        bool dead = false;
+        if (PASS_B) {
+            for (int r = threadIdx.x; r < MB * 128; r += kSoftThreads)
+                mp[r] = r < rows ? mprime[(size_t)u * kMaxRows + r] : INFINITY;
+            soft_barrier();
+        }
+        float m_run[MB], l_run[MB];
+#pragma unroll
+        for (int mb = 0; mb < MB; ++mb) { m_run[mb] = -INFINITY; l_run[mb] = 0.f; }
+
+        for (int i = 0; i < ntiles; ++i) {
+            const int tile_t0 = t0 + i * kTile;
+            float acc = 0.f;
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) {
+                const int q = i * MB + mb, buf = q % kNB;
+                uint32_t v[64];
+                if (!dead) {
+                    const bool ok = tc::mbar_wait(tc::smem_u32(&T.tfull[buf]), (q / kNB) & 1, status);
+                    dead = !__all_sync(0xffffffffu, ok);
+                }
+                if (!dead) {
+                    tc::tc_fence_after();
+                    uint32_t va[32], vb[32];
+                    tc::tmem_ld32(tbase + buf * 128, va);
+                    tc::tmem_ld32(tbase + buf * 128 + 32, vb);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) { v[j] = va[j]; v[32 + j] = vb[j]; }
+                    tc::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) tc::mbar_arrive(tc::smem_u32(&T.tempty[buf]));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) v[j] = 0u;
+                }
+                if (PASS_B) {
+                    const float *mrow = mp + mb * 128 + hf * 64;
+#pragma unroll
+                    for (int j = 0; j < 64; j += 4) {
+                        const float4 m4 = *reinterpret_cast<const float4 *>(mrow + j);
+                        acc += ex2(fmaf(__uint_as_float(v[j]), c_log2, -m4.x));
+                        acc += ex2(fmaf(__uint_as_float(v[j + 1]), c_log2, -m4.y));
+                        acc += ex2(fmaf(__uint_as_float(v[j + 2]), c_log2, -m4.z));
+                        acc += ex2(fmaf(__uint_as_float(v[j + 3]), c_log2, -m4.w));
+                    }
+                } else {
+                    const int r = mb * 128 + lane_row;
+                    const int last = P + (r % w);                       // last visible position of this row
+                    const int pos0 = tile_t0 + hf * 64;
+                    const bool masked = tile_t0 + kTile > P;            // uniform over the CTA
+#pragma unroll
+                    for (int piece = 0; piece < 2; ++piece) {
+                        float x[32];
+                        float pm = -INFINITY;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            x[j] = __uint_as_float(v[piece * 32 + j]);
+                            if (masked && pos0 + piece * 32 + j > last) x[j] = -INFINITY;
+                            pm = fmaxf(pm, x[j]);
+                        }
+                        const float m_new = fmaxf(m_run[mb], pm * c_log2);
+                        if (m_new > -INFINITY) {
+                            float sum = 0.f;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) sum += ex2(fmaf(x[j], c_log2, -m_new));
+                            l_run[mb] = l_run[mb] * ex2(m_run[mb] - m_new) + sum;
+                            m_run[mb] = m_new;
+                        }
+                    }
+                }
+            }
+            if (PASS_B) {
+                float *cs = colsum + (i & 1) * 256;
+                cs[hf * 128 + lane_row] = acc;
+                soft_barrier();
+                const int pos = tile_t0 + lane_row;
+                if (hf == 0 && pos < t1 && !dead) raw[(size_t)u * P + pos] = cs[lane_row] + cs[128 + lane_row];
+            }
+        }
+        if (!PASS_B && !dead) {
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) {
+                const int r = mb * 128 + lane_row;
+                if (r < rows) {
+                    float *o = stats_part + (((size_t)u * (2 * splits) + 2 * c + hf) * kMaxRows + r) * 2;
+                    o[0] = m_run[mb];
+                    o[1] = l_run[mb];
+                }
+            }
+        }
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 9) tc::tmem_dealloc(tmem, 512);
+}
+
+// one thread per (unit, row): partial (m, l) in index order -> m' = m + log2 l
+__global__ void score_tc_merge_kernel(const float *__restrict__ stats_part, int units, int rows, int parts,
+                                      float *__restrict__ mprime) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= units * rows) return;
+    const int u = idx / rows, r = idx % rows;
+    float m = -INFINITY;
+    for (int p = 0; p < parts; ++p) m = fmaxf(m, stats_part[(((size_t)u * parts + p) * kMaxRows + r) * 2]);
+    float l = 0.f;
+    for (int p = 0; p < parts; ++p) {
+        const float *s = stats_part + (((size_t)u * parts + p) * kMaxRows + r) * 2;
+        if (s[0] > -INFINITY) l += s[1] * exp2f(s[0] - m);
+    }
+    mprime[(size_t)u * kMaxRows + r] = m + log2f(l);
+}
+
+template <int MB>
+static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, const CUtensorMap &tk, float c_log2,
+                                       float *d_stats_part, float *d_mprime, float *d_raw, uint32_t *d_status,
+                                       Profiler *prof, cudaStream_t st) {
+    const uncomp_shape &s = p.shape;
+    const int smem = score_smem(MB);
+    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<MB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(score_tc_kernel<MB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    {
+        ProfScope ps(prof, kSlotScoreStats, st);
+        dim3 grid(p.score_splits, p.units);
+        score_tc_kernel<MB, false><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
+                                                                      p.score_splits, c_log2, d_stats_part, nullptr,
+                                                                      nullptr, d_status);
+    }
+    {
+        ProfScope ps(prof, kSlotStatsMerge, st);
+        const int total = p.units * p.rows;
+        score_tc_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows, 2 * p.score_splits,
+                                                                   d_mprime);
+    }
+    {
+        ProfScope ps(prof, kSlotScoreColsum, st);
+        const int splitsB = (p.prefix + p.score_chunk - 1) / p.score_chunk;
+        dim3 grid(splitsB, p.units);
+        score_tc_kernel<MB, true><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
+                                                                     splitsB, c_log2, nullptr, d_mprime, d_raw,
+                                                                     d_status);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
+                             float *d_stats_part, float *d_stats, float *d_raw, uint32_t *d_status, Profiler *prof,
+                             cudaStream_t st) {
+    CUtensorMap tq, tk;
+    cudaError_t e = make_query_tensor_map(&tq, dQw, p.units, p.rows);
+    if (e != cudaSuccess) return e;
+    e = make_key_tensor_map(&tk, p.shape, addr, dK, kTile);
+    if (e != cudaSuccess) return e;
+    const float c_log2 = scale * 1.4426950408889634f;
+    const int MB = (p.rows + 127) / 128;
+    switch (MB) {
+        case 1: return launch_scores_tc_mb<1>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_status, prof, st);
+        case 2: return launch_scores_tc_mb<2>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_status, prof, st);
+        case 3: return launch_scores_tc_mb<3>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_status, prof, st);
+        default: return launch_scores_tc_mb<4>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_status, prof, st);
+    }
+}
+
+}  // namespace uncomp

@@ -139,4 +139,8 @@ cudaError_t encode_tensor_map(CUtensorMap *map, const void *base, int rank, cons
                               const uint64_t *strides_bytes, const uint32_t *box, CUtensorMapDataType dtype,
                               CUtensorMapSwizzle swizzle);
 
+cudaError_t make_key_tensor_map(CUtensorMap *map, const uncomp_shape &s, const UnitAddr &addr, const void *dK,
+                                int tile_tokens);
+cudaError_t make_query_tensor_map(CUtensorMap *map, const void *dQw, int units, int rows);
+
 }  // namespace uncomp

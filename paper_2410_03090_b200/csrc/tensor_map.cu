@@ -30,4 +30,27 @@ cudaError_t encode_tensor_map(CUtensorMap *map, const void *base, int rank, cons
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// Tensor map over bf16 keys [B, L, H, N, d] with arbitrary (16-byte aligned) strides: dimensions
+// (feature, token, head, layer, batch), box = 64 features x tile_tokens tokens, 128-byte swizzle.
+// Tokens beyond N read as zero.
+cudaError_t make_key_tensor_map(CUtensorMap *map, const uncomp_shape &s, const UnitAddr &addr, const void *dK,
+                                int tile_tokens) {
+    uint64_t dims[5] = {(uint64_t)s.d, (uint64_t)s.N, (uint64_t)s.H, (uint64_t)s.L, (uint64_t)s.B};
+    uint64_t str[4] = {(uint64_t)addr.sN * 2, (uint64_t)addr.sH * 2, (uint64_t)addr.sL * 2, (uint64_t)addr.sB * 2};
+    // a dimension of extent 1 may come with stride 0: give it a harmless valid stride
+    for (int i = 0; i < 4; ++i)
+        if (dims[i + 1] == 1 && str[i] == 0) str[i] = (i == 0 ? (uint64_t)s.d * 2 : str[i - 1] * dims[i]);
+    uint32_t box[5] = {64, (uint32_t)tile_tokens, 1, 1, 1};
+    return encode_tensor_map(map, dK, 5, dims, str, box, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+// Tensor map over the window queries [units, rows, d] (contiguous bf16): box = 64 features x 128 rows.
+// Rows beyond `rows` read as zero.
+cudaError_t make_query_tensor_map(CUtensorMap *map, const void *dQw, int units, int rows) {
+    uint64_t dims[3] = {(uint64_t)kD, (uint64_t)rows, (uint64_t)units};
+    uint64_t str[2] = {(uint64_t)kD * 2, (uint64_t)rows * kD * 2};
+    uint32_t box[3] = {64, 128, 1};
+    return encode_tensor_map(map, dQw, 3, dims, str, box, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
 }  // namespace uncomp

@@ -292,3 +292,23 @@ def test_gram_tensor_core_vs_cuda_core_and_oracle():
         got = g_tc[u].cpu().numpy()
         assert np.abs(got[:128 * 128].reshape(128, 128) - G).max() <= 2e-6 * np.abs(G).max()
         assert np.abs(got[128 * 128:] - s).max() <= 2e-6 * np.abs(np.diag(G)).max() ** 0.5 * wl.N ** 0.5 + 1e-3
+
+
+@pytest.mark.parametrize("name,N", [("c2", 3000), ("c3", 4500), ("c5", 2100)])
+def test_scorer_tensor_core_vs_cuda_core(name, N):
+    # the two implementations of the same definition must agree far inside the oracle tolerance
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS[name], N=N, L=1)
+    K, V, Qw = synth.generate(wl, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    er = torch.ones(wl.B, wl.L, wl.H, device="cuda")
+    b, o, _, _ = ub.uncomp_assign_budgets(ctx, er, wl.avg_budget, 1, wl.avg_budget)
+    s_tc = torch.empty(wl.B, wl.L, wl.H, N - wl.w, device="cuda")
+    s_cc = torch.empty_like(s_tc)
+    ub.uncomp_score_select(ctx, Qw, K, b, o, wl.total_rows, 1, 0, 0.0, s_tc)
+    ub.uncomp_set_option(ctx, ub.UNCOMP_OPT_CUDA_CORES, 1)
+    ub.uncomp_score_select(ctx, Qw, K, b, o, wl.total_rows, 1, 0, 0.0, s_cc)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    rel = ((s_tc - s_cc).abs() / (s_cc.abs() + 1e-12 * s_cc.amax(dim=-1, keepdim=True))).max()
+    assert float(rel) < 5e-4, float(rel)
