@@ -201,6 +201,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--scale-N", type=int, default=0, help="profiling aid: same recipe at a shorter sequence")
+    ap.add_argument("--scale-L", type=int, default=0, help="profiling aid: same recipe with fewer layers")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -227,6 +229,8 @@ def main():
         dist.init_process_group(backend="nccl", device_id=dev)
 
     base = synth.WORKLOADS[args.workload]
+    if args.scale_N or args.scale_L:
+        base = synth.scaled(base, N=args.scale_N or None, L=args.scale_L or None)
     wl = replace(base, seed=base.seed + 7919 * rank)      # every rank compresses its own sequence(s)
     peaks = _peaks()
     K, V, Qw = synth.generate(wl, dev)
