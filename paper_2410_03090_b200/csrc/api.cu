@@ -232,7 +232,10 @@ int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const un
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     {
         ProfScope ps(ctx->prof, kSlotEigen, st);
-        e = launch_eigen_entropy(p, partials, *params, d_entropy, d_erank, d_spectrum, d_status, st);
+        if (p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt)
+            e = launch_eigen_f32(p, partials, *params, d_entropy, d_erank, d_spectrum, d_status, st);
+        else
+            e = launch_eigen_entropy(p, partials, *params, d_entropy, d_erank, d_spectrum, d_status, st);
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;

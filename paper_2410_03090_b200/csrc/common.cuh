@@ -77,6 +77,8 @@ cudaError_t launch_gram_tc(const Plan &p, const void *dK, const UnitAddr &addr, 
 cudaError_t launch_eigen_entropy(const Plan &p, const void *d_partials, const uncomp_entropy_params &ep,
                                  float *d_entropy, float *d_erank, double *d_spectrum, uint32_t *d_status,
                                  cudaStream_t st);
+cudaError_t launch_eigen_f32(const Plan &p, const void *d_partials, const uncomp_entropy_params &ep, float *d_entropy,
+                             float *d_erank, double *d_spectrum, uint32_t *d_status, cudaStream_t st);
 cudaError_t launch_gram_reduce(const Plan &p, const void *d_partials, double *d_out, cudaStream_t st);
 int check_budget_params(const uncomp_shape &s, const uncomp_budget_params &bp);
 cudaError_t launch_budgets(const Plan &p, const float *d_erank, const uncomp_budget_params &bp, int32_t *d_budgets,

@@ -312,3 +312,22 @@ def test_scorer_tensor_core_vs_cuda_core(name, N):
     assert ub.uncomp_status(ctx) == 0
     rel = ((s_tc - s_cc).abs() / (s_cc.abs() + 1e-12 * s_cc.amax(dim=-1, keepdim=True))).max()
     assert float(rel) < 5e-4, float(rel)
+
+
+def test_bf16_spectrum_register_kernel_vs_oracle():
+    # bf16 keys take the fp32 register-resident eigen kernel: its top-k spectrum against the oracle's
+    # Jacobi eigenvalues (tolerance of an fp32 reduction: 2e-6 of the largest eigenvalue)
+    import oracle
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c5"], N=3000, L=2)
+    K, _, _ = synth.generate(wl, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    spec = torch.empty(wl.B, wl.L, wl.H, 128, dtype=torch.float64, device="cuda")
+    ent, er = ub.uncomp_entropy(ctx, K, k_trunc=128, norm=1, spectrum=spec)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    for u in range(0, wl.units, 3):
+        H, E, lam = oracle.entropy(parity.unit_np(K, wl, u), k_trunc=128, norm=1, return_spectrum=True)
+        got = spec.reshape(-1, 128)[u].cpu().numpy()
+        np.testing.assert_allclose(got, lam, rtol=0, atol=2e-6 * lam[0])
+        assert abs(float(ent.reshape(-1)[u]) - H) <= 1e-4 * max(abs(H), 1.0)
