@@ -4,16 +4,18 @@
 // Two kernels with one pipeline skeleton; softmax needs the row statistics before the column sums:
 //   pass A  S = Qw K^T with the window rows on the TMEM lanes (M = 128 rows, N = 128 tokens per MMA tile):
 //           a thread owns a row, so its running maximum and sum of exponentials are thread-local;
-//           every (unit, chunk, column half) writes partial statistics (m, l) in the log2 domain;
+//           every (unit, chunk) writes partial statistics (m, l) in the log2 domain;
 //   merge   partials combined in index order into m'_r = m_r + log2 l_r;
 //   pass B  operands swapped (M = 128 tokens on the lanes, N = 128 rows): a thread owns a token and adds
 //           2^(s c - m'_r) along its TMEM row; tokens of a warp are consecutive, the store is coalesced.
 // K tiles (128 tokens x 128 features, two 128B-swizzled boxes of 64 features) stream through a TMA ring;
 // the unit's window queries stay in shared memory for the whole CTA.  Both operands are K-major.
 //
-// CTA = 320 threads on one SM: warps 0-7 softmax (warp % 4 selects the TMEM lane quarter, warp / 4 the
-// column half of an accumulator), warp 8 TMA producer, warp 9 TMEM allocation and MMA issue.  Four
-// 128-column accumulators rotate, so the tensor pipe runs ahead of the exponentials.
+// CTA = 576 threads on one SM: warps 0-15 softmax in two groups of eight that take alternate token tiles
+// (so the four warps of an SM sub-partition are in different phases: while one group waits for its
+// accumulator, the other keeps the exponential unit busy); inside a group warp % 4 selects the TMEM lane
+// quarter and bit 2 of the warp index the 64-column half of an accumulator.  Warp 16 is the TMA producer,
+// warp 17 allocates TMEM and issues the MMAs.  Each group owns two of the four 128-column accumulators.
 // Every wait is bounded; a timeout raises UNCOMP_STATUS_TIMEOUT and the CTA drains and exits.
 #include "tc_common.cuh"
 
@@ -24,7 +26,7 @@ constexpr int kTile = 128;
 constexpr int kHalfBytes = 128 * 128;            // 64 features x 128 rows/tokens, bf16
 constexpr int kBlockBytes = 2 * kHalfBytes;      // one K tile or one block of 128 query rows
 constexpr int kNB = 4;                           // accumulator buffers (x 128 TMEM columns = all 512)
-constexpr int kSoftThreads = 256;
+constexpr int kSoftThreads = 512;
 constexpr int kScoreThreads = kSoftThreads + 64;
 constexpr int kMaxStages = 4;
 
@@ -35,7 +37,7 @@ struct ScoreTail {
 
 __host__ __device__ constexpr int score_stages(int MB) { return MB <= 2 ? 4 : (MB == 3 ? 3 : 2); }
 __host__ __device__ constexpr int score_smem(int MB) {
-    return 1024 + MB * kBlockBytes + score_stages(MB) * kBlockBytes + MB * 128 * 4 + 2 * 2 * 128 * 4 +
+    return 1024 + MB * kBlockBytes + score_stages(MB) * kBlockBytes + MB * 128 * 4 + 2 * 4 * 128 * 4 +
            (int)sizeof(ScoreTail);
 }
 
@@ -44,7 +46,58 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void soft_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void all_soft_barrier() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
+__device__ __forceinline__ void group_barrier(int g) { asm volatile("bar.sync %0, 256;" ::"r"(1 + g) : "memory"); }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// Pass A: fold 64 logits of one row into its running (m, l), log2 domain.  m only has to stay at or above
+// every logit seen so far (it is the exact running maximum here, raised lazily), l = sum 2^(x c - m).
+template <bool MASKED>
+__device__ __forceinline__ void stats_update(uint32_t (&v)[64], float c_log2, int pos0, int last, float &m_run,
+                                             float &l_run) {
+    if (MASKED) {
+#pragma unroll
+        for (int j = 0; j < 64; ++j)
+            if (pos0 + j > last) v[j] = 0xff800000u;            // -inf: not visible to this row
+    }
+    float pm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+    for (int j = 0; j < 64; j += 8) {
+        pm[0] = max3(pm[0], __uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+        pm[1] = max3(pm[1], __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+        pm[2] = max3(pm[2], __uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
+        pm[3] = max3(pm[3], __uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
+    }
+    const float mx = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3])) * c_log2;
+    if (mx > m_run) {                                           // rare after the first tiles
+        l_run *= ex2(m_run - mx);
+        m_run = mx;
+    }
+    if (m_run > -INFINITY) {
+        float sum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int j = 0; j < 64; ++j) sum[j & 3] += ex2(fmaf(__uint_as_float(v[j]), c_log2, -m_run));
+        l_run += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+    }
+}
+
+// Pass B: sum over 64 window rows of 2^(s c - m'_r) for one token.
+__device__ __forceinline__ float colsum_partial(const uint32_t (&v)[64], float c_log2, const float *mrow) {
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int j = 0; j < 64; j += 4) {
+        const float4 m4 = *reinterpret_cast<const float4 *>(mrow + j);
+        acc[0] += ex2(fmaf(__uint_as_float(v[j]), c_log2, -m4.x));
+        acc[1] += ex2(fmaf(__uint_as_float(v[j + 1]), c_log2, -m4.y));
+        acc[2] += ex2(fmaf(__uint_as_float(v[j + 2]), c_log2, -m4.z));
+        acc[3] += ex2(fmaf(__uint_as_float(v[j + 3]), c_log2, -m4.w));
+    }
+    return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+}
 }  // namespace
 
 template <int MB, bool PASS_B>
@@ -60,8 +113,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
     const uint32_t q_addr = raw_addr + pad;
     const uint32_t k_addr = q_addr + MB * kBlockBytes;
     float *mp = reinterpret_cast<float *>(smem + (MB + S) * kBlockBytes);      // [MB * 128]
-    float *colsum = mp + MB * 128;                                             // [2][2][128]
-    ScoreTail &T = *reinterpret_cast<ScoreTail *>(colsum + 2 * 2 * 128);
+    float *colsum = mp + MB * 128;                                             // [2][4][128]
+    ScoreTail &T = *reinterpret_cast<ScoreTail *>(colsum + 2 * 4 * 128);
 
     const int c = blockIdx.x, u = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -80,15 +133,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
         tc::mbar_init(tc::smem_u32(&T.qfull), 1);
         for (int i = 0; i < kNB; ++i) {
             tc::mbar_init(tc::smem_u32(&T.tfull[i]), 1);
-            tc::mbar_init(tc::smem_u32(&T.tempty[i]), kSoftThreads / 32);
+            tc::mbar_init(tc::smem_u32(&T.tempty[i]), kSoftThreads / 64);   // the 8 warps of one group
         }
         tc::fence_mbar_init();
     }
-    if (warp == 9) {
+    if (warp == 17) {
         tc::tmem_alloc(tc::smem_u32(&T.tmem_base), 512);
         tc::tmem_relinquish();
     }
-    if (warp == 8 && lane == 0) {
+    if (warp == 16 && lane == 0) {
         tc::prefetch_tmap(&tmapQ);
         tc::prefetch_tmap(&tmapK);
     }
@@ -97,7 +150,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
     tc::tc_fence_after();
     const uint32_t tmem = T.tmem_base;
 
-    if (warp == 8) {
+    if (warp == 16) {
         // ---------------- TMA producer ----------------
         if (lane == 0 && ntiles > 0) {
             const uint32_t qbar = tc::smem_u32(&T.qfull);
@@ -124,7 +177,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                     tc::mbar_wait(tc::smem_u32(&T.full[i % S]), (i / S) & 1, status);
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == 17) {
         // ---------------- MMA issue ----------------
         if (lane == 0 && ntiles > 0) {
             constexpr uint32_t idesc = tc::idesc_bf16_f32(128, 128, 0, 0);
@@ -135,8 +188,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                 if (!ok) break;
                 const uint32_t kbase = k_addr + s * kBlockBytes;
                 for (int mb = 0; mb < MB && ok; ++mb) {
-                    const int q = i * MB + mb, buf = q % kNB;
-                    if (q >= kNB) ok = tc::mbar_wait(tc::smem_u32(&T.tempty[buf]), ((q / kNB) - 1) & 1, status);
+                    // each softmax group owns two accumulators: tile i belongs to group i & 1
+                    const int lq = (i >> 1) * MB + mb, buf = 2 * (i & 1) + (lq & 1);
+                    if (lq >= 2) ok = tc::mbar_wait(tc::smem_u32(&T.tempty[buf]), ((lq >> 1) - 1) & 1, status);
                     if (!ok) break;
                     tc::tc_fence_after();
                     const uint32_t qbase = q_addr + mb * kBlockBytes;
@@ -156,28 +210,29 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
         }
     } else {
         // ---------------- softmax warps ----------------
-        const int quarter = warp & 3, hf = warp >> 2;
+        const int quarter = warp & 3, half = (warp >> 2) & 1, group = warp >> 3;
         const int lane_row = quarter * 32 + lane;          // TMEM lane: a window row (A) or a token (B)
-        const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)hf * 64;
+        const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)half * 64;
         bool dead = false;
         if (PASS_B) {
             for (int r = threadIdx.x; r < MB * 128; r += kSoftThreads)
                 mp[r] = r < rows ? mprime[(size_t)u * kMaxRows + r] : INFINITY;
-            soft_barrier();
+            all_soft_barrier();
         }
         float m_run[MB], l_run[MB];
 #pragma unroll
         for (int mb = 0; mb < MB; ++mb) { m_run[mb] = -INFINITY; l_run[mb] = 0.f; }
 
-        for (int i = 0; i < ntiles; ++i) {
+        for (int i = group; i < ntiles; i += 2) {           // this group's tiles
             const int tile_t0 = t0 + i * kTile;
+            const bool masked = tile_t0 + kTile > P;            // uniform over the CTA
             float acc = 0.f;
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
-                const int q = i * MB + mb, buf = q % kNB;
+                const int lq = (i >> 1) * MB + mb, buf = 2 * group + (lq & 1);
                 uint32_t v[64];
                 if (!dead) {
-                    const bool ok = tc::mbar_wait(tc::smem_u32(&T.tfull[buf]), (q / kNB) & 1, status);
+                    const bool ok = tc::mbar_wait(tc::smem_u32(&T.tfull[buf]), (lq >> 1) & 1, status);
                     dead = !__all_sync(0xffffffffu, ok);
                 }
                 if (!dead) {
@@ -196,64 +251,56 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                     for (int j = 0; j < 64; ++j) v[j] = 0u;
                 }
                 if (PASS_B) {
-                    const float *mrow = mp + mb * 128 + hf * 64;
-#pragma unroll
-                    for (int j = 0; j < 64; j += 4) {
-                        const float4 m4 = *reinterpret_cast<const float4 *>(mrow + j);
-                        acc += ex2(fmaf(__uint_as_float(v[j]), c_log2, -m4.x));
-                        acc += ex2(fmaf(__uint_as_float(v[j + 1]), c_log2, -m4.y));
-                        acc += ex2(fmaf(__uint_as_float(v[j + 2]), c_log2, -m4.z));
-                        acc += ex2(fmaf(__uint_as_float(v[j + 3]), c_log2, -m4.w));
-                    }
+                    acc += colsum_partial(v, c_log2, mp + mb * 128 + half * 64);
                 } else {
                     const int r = mb * 128 + lane_row;
                     const int last = P + (r % w);                       // last visible position of this row
-                    const int pos0 = tile_t0 + hf * 64;
-                    const bool masked = tile_t0 + kTile > P;            // uniform over the CTA
-#pragma unroll
-                    for (int piece = 0; piece < 2; ++piece) {
-                        float x[32];
-                        float pm = -INFINITY;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            x[j] = __uint_as_float(v[piece * 32 + j]);
-                            if (masked && pos0 + piece * 32 + j > last) x[j] = -INFINITY;
-                            pm = fmaxf(pm, x[j]);
-                        }
-                        const float m_new = fmaxf(m_run[mb], pm * c_log2);
-                        if (m_new > -INFINITY) {
-                            float sum = 0.f;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) sum += ex2(fmaf(x[j], c_log2, -m_new));
-                            l_run[mb] = l_run[mb] * ex2(m_run[mb] - m_new) + sum;
-                            m_run[mb] = m_new;
-                        }
-                    }
+                    const int pos0 = tile_t0 + half * 64;
+                    if (masked) stats_update<true>(v, c_log2, pos0, last, m_run[mb], l_run[mb]);
+                    else stats_update<false>(v, c_log2, pos0, last, m_run[mb], l_run[mb]);
                 }
             }
             if (PASS_B) {
-                float *cs = colsum + (i & 1) * 256;
-                cs[hf * 128 + lane_row] = acc;
-                soft_barrier();
+                // the two column halves of this group meet in shared memory (slot = tile parity within the group)
+                float *cs = colsum + ((i >> 1) & 1) * 512 + group * 256;
+                cs[half * 128 + lane_row] = acc;
+                group_barrier(group);
                 const int pos = tile_t0 + lane_row;
-                if (hf == 0 && pos < t1 && !dead) raw[(size_t)u * P + pos] = cs[lane_row] + cs[128 + lane_row];
+                if (half == 0 && pos < t1 && !dead) raw[(size_t)u * P + pos] = cs[lane_row] + cs[128 + lane_row];
             }
         }
-        if (!PASS_B && !dead) {
+        if (!PASS_B) {
+            // merge the four (group, half) partials of every row in a fixed order; the K stages are idle by now
+            float2 *merge = reinterpret_cast<float2 *>(smem + MB * kBlockBytes);      // [4][MB * 128]
+            const int slot = group * 2 + half;
 #pragma unroll
-            for (int mb = 0; mb < MB; ++mb) {
-                const int r = mb * 128 + lane_row;
-                if (r < rows) {
-                    float *o = stats_part + (((size_t)u * (2 * splits) + 2 * c + hf) * kMaxRows + r) * 2;
-                    o[0] = m_run[mb];
-                    o[1] = l_run[mb];
+            for (int mb = 0; mb < MB; ++mb) merge[slot * (MB * 128) + mb * 128 + lane_row] = make_float2(m_run[mb], l_run[mb]);
+            all_soft_barrier();
+            if (slot == 0 && !dead) {
+#pragma unroll
+                for (int mb = 0; mb < MB; ++mb) {
+                    const int r = mb * 128 + lane_row;
+                    if (r < rows) {
+                        float m = -INFINITY;
+#pragma unroll
+                        for (int sl = 0; sl < 4; ++sl) m = fmaxf(m, merge[sl * (MB * 128) + r].x);
+                        float lsum = 0.f;
+#pragma unroll
+                        for (int sl = 0; sl < 4; ++sl) {
+                            const float2 ml = merge[sl * (MB * 128) + r];
+                            if (ml.x > -INFINITY) lsum += ml.y * ex2(ml.x - m);
+                        }
+                        float *o = stats_part + (((size_t)u * splits + c) * kMaxRows + r) * 2;
+                        o[0] = m;
+                        o[1] = lsum;
+                    }
                 }
             }
         }
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 9) tc::tmem_dealloc(tmem, 512);
+    if (warp == 17) tc::tmem_dealloc(tmem, 512);
 }
 
 // one thread per (unit, row): partial (m, l) in index order -> m' = m + log2 l
@@ -292,7 +339,7 @@ static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, con
     {
         ProfScope ps(prof, kSlotStatsMerge, st);
         const int total = p.units * p.rows;
-        score_tc_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows, 2 * p.score_splits,
+        score_tc_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows, p.score_splits,
                                                                    d_mprime);
     }
     {
