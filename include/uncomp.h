@@ -120,6 +120,31 @@ int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const un
  * d_gram  out  [B*L*H, d*d + d] double: G row-major, then s. */
 int uncomp_gram(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, double *d_gram, void *stream);
 
+/* uncomp_gram_static -- uncomp_gram for callers that cannot allocate device memory.  The paper has no
+ * counterpart: this entry point exists for integration only.
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits, and that therefore cannot create the
+ * workspace every other call of this library lives in -- a custom-operator hook inside a serving framework
+ * whose own caching allocator owns the device memory, or a latency-critical thread that must not take the
+ * device-wide stall an allocation or a free causes.  It needs no context and no workspace: the per-chunk
+ * partial sums go to a fixed array inside the library image (uncomp_gram_static_max_bytes() = 4,227,072
+ * bytes, plus one status word), which every GPU that loads the library holds until the process exits.
+ * The call itself allocates nothing, on the device or through any library.
+ *
+ * Limits and rules
+ *   - (units) x (token chunks per unit) partials must fit the array: at most 64 partials for bf16 keys,
+ *     32 for fp32 keys (e.g. 8 heads x 32768 tokens in bf16 is 8 x 8 = 64).  Larger shapes are refused
+ *     with UNCOMP_E_LIMIT and nothing is launched.
+ *   - The first call on a device looks up the array's device address (the device must be current).  Make
+ *     that first call outside any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents; this call overwrites the
+ *     part it reads and clears its status word itself.  Two calls whose GPU work overlaps (different
+ *     streams, or threads) race on it: serialise them.
+ *   - Device-side conditions (a bounded wait that expired) are not reported by this entry point.
+ * Arguments as for uncomp_gram, with the shape passed directly; the result is identical to uncomp_gram's. */
+int uncomp_gram_static(const uncomp_shape *shape, const void *d_K, uncomp_strides sK, double *d_gram, void *stream);
+size_t uncomp_gram_static_max_bytes(void);
+
 /* ---------------------------------------------------------------------------------------------------
  * uncomp_assign_budgets -- Section 3.3.3 "Head-Group Compression": heads ranked by truncated effective
  * rank, split into M groups, group budgets N_{i,g+1} = N_{i,g} - step from n_max downwards; and

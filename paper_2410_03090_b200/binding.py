@@ -63,6 +63,9 @@ def _load() -> C.CDLL:
     lib.uncomp_entropy.argtypes = [vp, vp, uncomp_strides, C.POINTER(uncomp_entropy_params), fp, fp, dp, vp]
     lib.uncomp_gram.restype = C.c_int
     lib.uncomp_gram.argtypes = [vp, vp, uncomp_strides, dp, vp]
+    lib.uncomp_gram_static.restype = C.c_int
+    lib.uncomp_gram_static.argtypes = [C.POINTER(uncomp_shape), vp, uncomp_strides, dp, vp]
+    lib.uncomp_gram_static_max_bytes.restype = C.c_size_t
     lib.uncomp_assign_budgets.restype = C.c_int
     lib.uncomp_assign_budgets.argtypes = [vp, fp, C.POINTER(uncomp_budget_params), i32p, i64p, i32p, i32p, vp]
     lib.uncomp_score_select.restype = C.c_int
@@ -172,6 +175,14 @@ def uncomp_gram(ctx: Context, K: torch.Tensor, gram: Optional[torch.Tensor] = No
     if gram is None:
         gram = torch.empty(s.B * s.L * s.H, s.d * s.d + s.d, dtype=torch.float64, device=K.device)
     _check(lib.uncomp_gram(ctx.handle, _ptr(K), strides_of(K), _ptr(gram), _stream(stream)), "uncomp_gram")
+    return gram
+
+
+def uncomp_gram_static(shape: uncomp_shape, K: torch.Tensor, gram: torch.Tensor, stream=None) -> torch.Tensor:
+    """uncomp_gram without a context or workspace (scratch lives in a fixed array inside the library).
+    `gram` is the caller's [units, d*d + d] float64 output; nothing is allocated here."""
+    _check(lib.uncomp_gram_static(C.byref(shape), _ptr(K), strides_of(K), _ptr(gram), _stream(stream)),
+           "uncomp_gram_static")
     return gram
 
 

@@ -27,6 +27,8 @@ struct Plan {
     size_t bytes;
 };
 
+Plan make_plan(const uncomp_shape &s);
+
 struct UnitAddr {
     int L, H;
     int64_t sB, sL, sH, sN;
