@@ -215,7 +215,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2410_03090_b200 import binding as ub
-    from paper_2410_03090_b200 import synth
+    from paper_2410_03090_b200 import shard, synth
     from paper_2410_03090_b200.compress import CompressionPass
 
     rank = int(os.environ.get("RANK", "0"))
@@ -231,7 +231,7 @@ def main():
     base = synth.WORKLOADS[args.workload]
     if args.scale_N or args.scale_L:
         base = synth.scaled(base, N=args.scale_N or None, L=args.scale_L or None)
-    wl = replace(base, seed=base.seed + 7919 * rank)      # every rank compresses its own sequence(s)
+    wl = shard.rank_workload(base, rank)      # every rank compresses its own sequence(s)
     peaks = _peaks()
     K, V, Qw = synth.generate(wl, dev)
     cp = CompressionPass(wl, dev)
@@ -262,13 +262,10 @@ def main():
     ms_total = ev0.elapsed_time(ev1)
     prof = ub.uncomp_profile_read(cp.ctx)
     ub.uncomp_profile_enable(cp.ctx, False)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = shard.max_over_ranks(ms_total, dev, world)
     ms_step = ms_total / args.steps
     tokens_step = wl.B * wl.N * world
-    value = tokens_step / (ms_step / 1e3)
+    value = shard.whole_job_tokens_per_s(wl, world, ms_step)
 
     # ---- per-kernel roofline, from the events the library recorded inside the timed region
     specs = kernel_specs(wl, peaks, sustained=True)
@@ -329,10 +326,7 @@ def main():
         torch.cuda.synchronize()
         barrier()
         ms_e = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms_e], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e = float(t.item())
+        ms_e = shard.max_over_ranks(ms_e, dev, world)
         e2e = {"value": tokens_step / (ms_e / args.e2e_steps / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
         del hK, hV, hQ, dK, dV, dQ

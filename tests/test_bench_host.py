@@ -1,0 +1,81 @@
+"""Host logic of the benchmark and of multi-GPU sharding, on CPU (gloo, world size 2)."""
+import json
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2410_03090_b200 import shard, synth
+    base = synth.scaled(synth.WORKLOADS["c2"], N=128, L=1)
+    wl = shard.rank_workload(base, rank)
+    K, _, _ = synth.generate_unit(wl, 0, 0, 0)
+    ms = shard.max_over_ranks(10.0 + 5.0 * rank, "cpu", world)          # the slowest rank decides
+    digest = torch.tensor([float(K.float().sum())], dtype=torch.float64)
+    gathered = [torch.zeros_like(digest) for _ in range(world)]
+    dist.all_gather(gathered, digest)
+    dist.barrier()
+    if rank == 0:
+        out.put({"ms": ms, "seed0": wl.seed, "digests": [float(g) for g in gathered],
+                 "value": shard.whole_job_tokens_per_s(wl, world, ms)})
+    dist.destroy_process_group()
+
+
+def test_two_ranks_shard_sequences_and_agree_on_time():
+    ctx = mp.get_context("spawn")
+    out = ctx.SimpleQueue()
+    port = 29000 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(120)
+        assert p.exitcode == 0
+    res = out.get()
+    assert res["ms"] == 15.0
+    assert res["digests"][0] != res["digests"][1]            # each rank compresses its own sequence
+    assert abs(res["value"] - 2 * 128 / 0.015) < 1e-6          # tokens of both ranks over the slowest time
+
+
+def test_rank_workload_keeps_shape_and_changes_data():
+    from paper_2410_03090_b200 import shard, synth
+    base = synth.WORKLOADS["c3"]
+    w0, w1 = shard.rank_workload(base, 0), shard.rank_workload(base, 1)
+    assert w0 == base and w1.seed != base.seed
+    assert (w1.N, w1.L, w1.H, w1.avg_budget, w1.n_max) == (base.N, base.L, base.H, base.avg_budget, base.n_max)
+    assert shard.max_over_ranks(3.5, "cpu", 1) == 3.5
+
+
+def test_reference_arm_prints_one_json_line_and_other_ranks_stay_silent():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                        "--warmup", "0", "--workload", "c1"], capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0 and r.stdout.strip() == ""
+    env["RANK"] = "0"
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                        "--warmup", "0", "--workload", "c1"], capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["value"] > 0 and line["unit"] == "tokens/s"
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+    assert line["higher_is_better"] is True and line["vs_baseline"] is None
+
+
+def test_kernel_specs_cover_every_profiled_kernel():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2410_03090_b200 import binding as ub, synth
+    specs = bench.kernel_specs(synth.WORKLOADS["c3"], bench._peaks(), True)
+    names = {ub.lib.uncomp_profile_slot_name(i).decode() for i in range(ub.lib.uncomp_profile_slots())}
+    assert names == set(specs)
+    # algorithmic work of the c3 pass: 0.275 TFLOP of Gram, 2.57 GB of bytes
+    assert abs(specs["gram"][1] - 0.2749) < 1e-3
+    assert abs(synth.WORKLOADS["c3"].algorithmic_bytes() / 1e9 - 2.5695) < 1e-3
