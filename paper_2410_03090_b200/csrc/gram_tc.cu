@@ -105,21 +105,24 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap tmap, int L, int H, int N, in
         if (lane == 0) {
             constexpr uint32_t idesc_g = tc::idesc_bf16_f32(128, 128, 1, 1);
             constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, 16, 1, 1);
+            // descriptors: MN-major, 128-byte swizzle; feature halves kRegion apart (LBO), 8-token groups
+            // 1024 B apart (SBO).  16 tokens further = 2048 B = +128 in the address field (16-byte units).
             const uint64_t ones_desc = tc::smem_desc_sw128(tiles_addr + kStages * kStageBytes, 1024, 1024);
+            const uint64_t tile_desc = tc::smem_desc_sw128(tiles_addr, kRegion, 1024);
+            const uint32_t dhi = tc::desc_hi(tile_desc), ones_hi = tc::desc_hi(ones_desc);
+            const uint32_t ones_lo = tc::desc_lo(ones_desc);
             bool ok = true;
             for (int i = 0; i < ntiles && ok; ++i) {
                 const int s = i % kStages;
                 ok = tc::mbar_wait(tc::smem_u32(&T.full[s]), (i / kStages) & 1, status);
                 if (!ok) { T.abort = 1; break; }
                 tc::tc_fence_after();
-                const uint32_t base = tiles_addr + s * kStageBytes;
+                const uint32_t lo = tc::desc_lo(tile_desc) + (uint32_t)(s * (kStageBytes >> 4));
 #pragma unroll
                 for (int k = 0; k < kTile / 16; ++k) {
-                    // 16 tokens further = 2048 B; feature halves kRegion apart (LBO), 8-token groups 1024 B (SBO)
-                    const uint64_t desc = tc::smem_desc_sw128(base + k * 2048, kRegion, 1024);
                     const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
-                    tc::mma_f16_ss(tmem, desc, desc, idesc_g, acc);
-                    tc::mma_f16_ss(tmem + 128, desc, ones_desc, idesc_s, acc);
+                    tc::mma_f16_ss_lohi(tmem, lo + k * 128, lo + k * 128, dhi, idesc_g, acc);
+                    tc::mma_f16_ss2(tmem + 128, lo + k * 128, dhi, ones_lo, ones_hi, idesc_s, acc);
                 }
                 tc::mma_commit(tc::smem_u32(&T.empty[s]));   // stage reusable once these MMAs have read it
             }

@@ -181,27 +181,34 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
         // ---------------- MMA issue ----------------
         if (lane == 0 && ntiles > 0) {
             constexpr uint32_t idesc = tc::idesc_bf16_f32(128, 128, 0, 0);
+            // descriptors: K-major, 128-byte swizzle, 8-row groups 1024 B apart.  Only the address field
+            // (16-byte units) of the lower half changes: +2 per 16 features inside a 128-byte row, +1024 for
+            // the second 64-feature half.
+            const uint64_t d0 = tc::smem_desc_sw128(q_addr, 16, 1024);
+            const uint32_t dhi = tc::desc_hi(d0);
+            uint32_t q_lo[MB];
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) q_lo[mb] = tc::desc_lo(d0) + (uint32_t)(mb * kBlockBytes >> 4);
+            const uint32_t k_lo0 = tc::desc_lo(tc::smem_desc_sw128(k_addr, 16, 1024));
             bool ok = tc::mbar_wait(tc::smem_u32(&T.qfull), 0, status);
             for (int i = 0; i < ntiles && ok; ++i) {
                 const int s = i % S;
                 ok = tc::mbar_wait(tc::smem_u32(&T.full[s]), (i / S) & 1, status);
                 if (!ok) break;
-                const uint32_t kbase = k_addr + s * kBlockBytes;
-                for (int mb = 0; mb < MB && ok; ++mb) {
+                const uint32_t k_lo = k_lo0 + (uint32_t)(s * (kBlockBytes >> 4));
+#pragma unroll
+                for (int mb = 0; mb < MB; ++mb) {
                     // each softmax group owns two accumulators: tile i belongs to group i & 1
                     const int lq = (i >> 1) * MB + mb, buf = 2 * (i & 1) + (lq & 1);
-                    if (lq >= 2) ok = tc::mbar_wait(tc::smem_u32(&T.tempty[buf]), ((lq >> 1) - 1) & 1, status);
+                    if (ok && lq >= 2) ok = tc::mbar_wait(tc::smem_u32(&T.tempty[buf]), ((lq >> 1) - 1) & 1, status);
                     if (!ok) break;
                     tc::tc_fence_after();
-                    const uint32_t qbase = q_addr + mb * kBlockBytes;
+                    const uint32_t d_tmem = tmem + buf * 128;
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        // 16 features further = 32 B inside the 128-byte swizzle row; second half one region on
-                        const uint32_t off = (uint32_t)(k >> 2) * kHalfBytes + (uint32_t)(k & 3) * 32;
-                        const uint64_t qd = tc::smem_desc_sw128(qbase + off, 16, 1024);
-                        const uint64_t kd = tc::smem_desc_sw128(kbase + off, 16, 1024);
-                        if (PASS_B) tc::mma_f16_ss(tmem + buf * 128, kd, qd, idesc, k > 0);
-                        else tc::mma_f16_ss(tmem + buf * 128, qd, kd, idesc, k > 0);
+                        const uint32_t off = (uint32_t)(k >> 2) * (kHalfBytes >> 4) + (uint32_t)(k & 3) * 2;
+                        if (PASS_B) tc::mma_f16_ss_lohi(d_tmem, k_lo + off, q_lo[mb] + off, dhi, idesc, k > 0);
+                        else tc::mma_f16_ss_lohi(d_tmem, q_lo[mb] + off, k_lo + off, dhi, idesc, k > 0);
                     }
                     tc::mma_commit(tc::smem_u32(&T.tfull[buf]));
                 }
