@@ -107,6 +107,7 @@ def kernel_specs(wl, peaks, sustained: bool):
     hbm = peaks["hbm_gbs"]
     return {
         "gram": ("tensor", 2.0 * N * d * d * u / 1e12, tens, "TFLOP/s"),
+        "gram_score_stats": ("tensor", (2.0 * N * d * d + 2.0 * rows * d * N) * u / 1e12, tens, "TFLOP/s"),
         "score_stats": ("tensor", 2.0 * rows * d * N * u / 1e12, tens, "TFLOP/s"),
         "score_colsum": ("tensor", 2.0 * rows * d * P * u / 1e12, tens, "TFLOP/s"),
         "pool_select": ("hbm", (2.0 * u * P * 4 + wl.total_rows * 4) / 1e9, hbm, "GB/s"),

@@ -99,7 +99,16 @@ void uncomp_destroy(uncomp_ctx *ctx);
  * unit that has not reached 1e-13 of its spectral radius by then sets UNCOMP_STATUS_NOT_CONVERGED
  * and still writes its current estimate.
  *
+ * Fusion with the scorer: the window scorer (uncomp_score_select) also sweeps over K and needs, before
+ * anything else, the softmax statistics of its window rows.  If d_Qw is given (bf16 keys only; ignored
+ * otherwise), those statistics are produced in the same sweep that forms the Gram matrices -- one read of
+ * K instead of two -- and are kept in the workspace.  The next uncomp_score_select call on this context
+ * with the same d_K, strides, d_Qw and scale then skips its statistics pass.  The caller must not change
+ * K or Qw in between.  d_Qw = NULL runs the entropy stage on its own.
+ *
  * d_K        in   [B, L, H, N, d] with strides sK, storage dtype of the shape
+ * d_Qw       in   [B, L, Hq, w, d] window queries as for uncomp_score_select, or NULL
+ * scale           logit scale of the scorer (0 means 1 / sqrt(d)); only used with d_Qw
  * d_entropy  out  [B, L, H] float, H_k
  * d_erank    out  [B, L, H] float, erank_k; may be NULL
  * d_spectrum out  [B, L, H, k] double, the k largest eigenvalues of C (unnormalised); may be NULL
@@ -112,7 +121,8 @@ typedef struct {
 } uncomp_entropy_params;
 
 int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const uncomp_entropy_params *params,
-                   float *d_entropy, float *d_erank, double *d_spectrum, void *stream);
+                   const void *d_Qw, float scale, float *d_entropy, float *d_erank, double *d_spectrum,
+                   void *stream);
 
 /* uncomp_gram -- the building blocks of Eq. 1 on their own: for every unit the Gram matrix G = X^T X and
  * the column sums s = X^T 1 (the covariance of Eq. 1 is (G - s s^T / N) / (N - 1)), as produced by the

@@ -60,7 +60,7 @@ def _load() -> C.CDLL:
     lib.uncomp_last_cuda_error.restype = C.c_int
     lib.uncomp_last_cuda_error.argtypes = [vp]
     lib.uncomp_entropy.restype = C.c_int
-    lib.uncomp_entropy.argtypes = [vp, vp, uncomp_strides, C.POINTER(uncomp_entropy_params), fp, fp, dp, vp]
+    lib.uncomp_entropy.argtypes = [vp, vp, uncomp_strides, C.POINTER(uncomp_entropy_params), vp, C.c_float, fp, fp, dp, vp]
     lib.uncomp_gram.restype = C.c_int
     lib.uncomp_gram.argtypes = [vp, vp, uncomp_strides, dp, vp]
     lib.uncomp_gram_static.restype = C.c_int
@@ -158,15 +158,17 @@ class Context:
 
 def uncomp_entropy(ctx: Context, K: torch.Tensor, k_trunc: int = 32, center: int = 1, norm: int = 0,
                    max_iters: int = 0, entropy: Optional[torch.Tensor] = None, erank: Optional[torch.Tensor] = None,
-                   spectrum: Optional[torch.Tensor] = None, stream=None):
+                   spectrum: Optional[torch.Tensor] = None, stream=None, Qw: Optional[torch.Tensor] = None,
+                   scale: float = 0.0):
+    """Qw given: the scorer's row statistics are produced in the same sweep over K (see uncomp.h)."""
     s = ctx.shape
     if entropy is None:
         entropy = torch.empty(s.B, s.L, s.H, dtype=torch.float32, device=K.device)
     if erank is None:
         erank = torch.empty(s.B, s.L, s.H, dtype=torch.float32, device=K.device)
     p = uncomp_entropy_params(k_trunc, center, norm, max_iters)
-    _check(lib.uncomp_entropy(ctx.handle, _ptr(K), strides_of(K), C.byref(p), _ptr(entropy), _ptr(erank),
-                              _ptr(spectrum), _stream(stream)), "uncomp_entropy")
+    _check(lib.uncomp_entropy(ctx.handle, _ptr(K), strides_of(K), C.byref(p), _ptr(Qw), scale, _ptr(entropy),
+                              _ptr(erank), _ptr(spectrum), _stream(stream)), "uncomp_entropy")
     return entropy, erank
 
 

@@ -27,8 +27,9 @@ class PassOutput:
 class CompressionPass:
     """Pre-allocates every output of a workload once; `run` launches the pass without host syncs."""
 
-    def __init__(self, wl: Workload, device: torch.device | str = "cuda"):
+    def __init__(self, wl: Workload, device: torch.device | str = "cuda", fused: bool = True):
         self.wl = wl
+        self.fused = fused    # entropy call also produces the scorer's row statistics (one sweep over K less)
         self.device = torch.device(device)
         self.shape = ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype)
         self.ctx = ub.Context(self.shape, self.device)
@@ -50,7 +51,7 @@ class CompressionPass:
     def run(self, K: torch.Tensor, V: torch.Tensor, Qw: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
             eps: float = 0.0, dn: int = 0, n_last: int = 0, scope: int = 0) -> PassOutput:
         wl, o, ctx = self.wl, self.out, self.ctx
-        ub.uncomp_entropy(ctx, K, wl.k_trunc, 1, 0, 0, o.entropy, o.erank, None, stream)
+        ub.uncomp_entropy(ctx, K, wl.k_trunc, 1, 0, 0, o.entropy, o.erank, None, stream, Qw=Qw if self.fused else None)
         ub.uncomp_assign_budgets(ctx, o.erank, wl.avg_budget, wl.M, wl.n_max, scope, eps, dn, n_last,
                                  o.budgets, o.offsets, o.layer_group, o.layer_ctx, stream)
         ub.uncomp_score_select(ctx, Qw, K, o.budgets, o.offsets, wl.total_rows, wl.pool_kernel, wl.pool_mode, 0.0,

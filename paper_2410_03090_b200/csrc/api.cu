@@ -39,8 +39,8 @@ Plan make_plan(const uncomp_shape &s) {
         p.gram_splits = (s.N + chunk - 1) / chunk;
     }
     {
-        // scorer: chunks of 4096 tokens (a multiple of the 128-token tile), halved while the grid is small
-        int chunk = 4096;
+        // scorer: chunks of 8192 tokens (a multiple of the 128-token tile), halved while the grid is small
+        int chunk = 8192;
         while (chunk > 512 && (int64_t)p.units * ((s.N + chunk - 1) / chunk) < target_ctas) chunk >>= 1;
         p.score_chunk = chunk;
         p.score_splits = (s.N + chunk - 1) / chunk;
@@ -48,7 +48,8 @@ Plan make_plan(const uncomp_shape &s) {
     const size_t acc = s.dtype == UNCOMP_FP32 ? sizeof(double) : sizeof(float);
     size_t o = 0;
     p.off_status = o;      o = align_up(o + 256, 256);
-    p.off_gram = o;        o = align_up(o + (size_t)p.units * p.gram_splits * (kD * kD + kD) * acc, 256);
+    const int gram_parts = p.gram_splits > p.score_splits ? p.gram_splits : p.score_splits;   // fused path: one per scorer chunk
+    p.off_gram = o;        o = align_up(o + (size_t)p.units * gram_parts * (kD * kD + kD) * acc, 256);
     p.off_stats_part = o;  o = align_up(o + (size_t)p.units * p.score_splits * 2 * kMaxRows * 2 * sizeof(float), 256);
     p.off_stats = o;       o = align_up(o + (size_t)p.units * kMaxRows * 2 * sizeof(float), 256);
     p.off_raw = o;         o = align_up(o + (size_t)p.units * p.prefix * sizeof(float), 256);
@@ -96,6 +97,11 @@ struct uncomp_ctx {
     Profiler *prof;   // NULL unless profiling is on
     Profiler prof_store;
     int force_simt;   // UNCOMP_OPT_CUDA_CORES
+    // row statistics left in the workspace by a fused uncomp_entropy call, valid for exactly these inputs
+    int stats_valid;
+    const void *stats_K, *stats_Qw;
+    uncomp_strides stats_sK;
+    float stats_scale;
 };
 
 static int cuda_fail(uncomp_ctx *ctx, cudaError_t e) {
@@ -153,6 +159,7 @@ int uncomp_create(uncomp_ctx **out, const uncomp_shape *shape, void *d_workspace
     ctx->device = 0;
     ctx->prof = nullptr;
     ctx->force_simt = 0;
+    ctx->stats_valid = 0;
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + p.off_status, 0, 256);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -187,7 +194,7 @@ int uncomp_profile_slots(void) { return kSlotCount; }
 
 const char *uncomp_profile_slot_name(int slot) {
     static const char *names[kSlotCount] = {"gram", "eigen_entropy", "budgets", "score_stats", "stats_merge",
-                                            "score_colsum", "pool_select", "compact"};
+                                            "score_colsum", "pool_select", "compact", "gram_score_stats"};
     return slot >= 0 && slot < kSlotCount ? names[slot] : "";
 }
 
@@ -209,31 +216,54 @@ int uncomp_profile_read(uncomp_ctx *ctx, int max_slots, float *ms_sum, int32_t *
 
 int uncomp_last_cuda_error(const uncomp_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
 
+static float effective_scale(float scale, int d) { return scale > 0.f ? scale : 1.0f / sqrtf((float)d); }
+
+static bool same_strides(const uncomp_strides &a, const uncomp_strides &b) {
+    return a.sB == b.sB && a.sL == b.sL && a.sH == b.sH && a.sN == b.sN;
+}
+
 int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const uncomp_entropy_params *params,
-                   float *d_entropy, float *d_erank, double *d_spectrum, void *stream) {
+                   const void *d_Qw, float scale, float *d_entropy, float *d_erank, double *d_spectrum,
+                   void *stream) {
     if (!ctx || !d_K || !params || !d_entropy) return UNCOMP_E_NULL;
     const Plan &p = ctx->plan;
-    if (!aligned16(d_K)) return UNCOMP_E_ALIGN;
+    if (!aligned16(d_K) || (d_Qw && !aligned16(d_Qw))) return UNCOMP_E_ALIGN;
     int rc = check_strides(p.shape, sK);
     if (rc != UNCOMP_OK) return rc;
     if (params->k_trunc < 1 || params->max_iters < 0 || (params->center != 0 && params->center != 1) ||
-        (params->norm != 0 && params->norm != 1))
+        (params->norm != 0 && params->norm != 1) || !(scale >= 0.f) || isinf(scale))
         return UNCOMP_E_PARAM;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint32_t *d_status = reinterpret_cast<uint32_t *>(ctx->ws + p.off_status);
     void *partials = ctx->ws + p.off_gram;
     const UnitAddr addr = make_addr(p.shape, sK);
+    const bool tensor_path = p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt;
+    ctx->stats_valid = 0;
     cudaError_t e;
-    {
+    int parts = p.gram_splits;
+    if (tensor_path && d_Qw) {
+        // one sweep over K: Gram partials per scorer chunk and the scorer's row statistics
+        const float sc = effective_scale(scale, p.shape.d);
+        e = launch_scores_tc(p, d_Qw, d_K, addr, sc, reinterpret_cast<float *>(ctx->ws + p.off_stats_part),
+                             reinterpret_cast<float *>(ctx->ws + p.off_stats), nullptr,
+                             reinterpret_cast<float *>(partials), kScorePhaseStats, d_status, ctx->prof, st);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        parts = p.score_splits;
+        ctx->stats_valid = 1;
+        ctx->stats_K = d_K;
+        ctx->stats_Qw = d_Qw;
+        ctx->stats_sK = sK;
+        ctx->stats_scale = sc;
+    } else {
         ProfScope ps(ctx->prof, kSlotGram, st);
-        if (p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt) e = launch_gram_tc(p, d_K, addr, partials, d_status, st);
+        if (tensor_path) e = launch_gram_tc(p, d_K, addr, partials, d_status, st);
         else e = launch_gram_simt(p, d_K, addr, partials, st);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
     }
-    if (e != cudaSuccess) return cuda_fail(ctx, e);
     {
         ProfScope ps(ctx->prof, kSlotEigen, st);
-        if (p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt)
-            e = launch_eigen_f32(p, partials, *params, d_entropy, d_erank, d_spectrum, d_status, st);
+        if (tensor_path)
+            e = launch_eigen_f32(p, partials, parts, *params, d_entropy, d_erank, d_spectrum, d_status, st);
         else
             e = launch_eigen_entropy(p, partials, *params, d_entropy, d_erank, d_spectrum, d_status, st);
     }
@@ -292,7 +322,7 @@ int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, unco
     if (params->pool_kernel < 1 || params->pool_kernel > 63 || (params->pool_kernel & 1) == 0 ||
         (params->pool_mode != 0 && params->pool_mode != 1) || !(params->scale >= 0.f) || isinf(params->scale))
         return UNCOMP_E_PARAM;
-    const float scale = params->scale > 0.f ? params->scale : 1.0f / sqrtf((float)p.shape.d);
+    const float scale = effective_scale(params->scale, p.shape.d);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint32_t *d_status = reinterpret_cast<uint32_t *>(ctx->ws + p.off_status);
     float *stats_part = reinterpret_cast<float *>(ctx->ws + p.off_stats_part);
@@ -301,10 +331,16 @@ int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, unco
     float *pooled = d_scores ? d_scores : reinterpret_cast<float *>(ctx->ws + p.off_pooled);
     const UnitAddr addr = make_addr(p.shape, sK);
     cudaError_t e;
-    if (p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt)
-        e = launch_scores_tc(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, d_status, ctx->prof, st);
-    else
+    if (p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt) {
+        // the statistics pass is skipped when a fused uncomp_entropy call left them for exactly these inputs
+        const bool reuse = ctx->stats_valid && ctx->stats_K == d_K && ctx->stats_Qw == d_Qw &&
+                           same_strides(ctx->stats_sK, sK) && ctx->stats_scale == scale;
+        ctx->stats_valid = 0;
+        const int phases = reuse ? kScorePhaseColsum : (kScorePhaseStats | kScorePhaseColsum);
+        e = launch_scores_tc(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, nullptr, phases, d_status, ctx->prof, st);
+    } else {
         e = launch_scores_simt(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, ctx->prof, st);
+    }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     {
         ProfScope ps(ctx->prof, kSlotPoolSelect, st);

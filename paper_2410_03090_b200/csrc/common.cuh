@@ -62,7 +62,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Optional per-kernel timing with CUDA events on the launching stream (host objects only).
 enum Slot { kSlotGram = 0, kSlotEigen, kSlotBudgets, kSlotScoreStats, kSlotStatsMerge, kSlotScoreColsum,
-            kSlotPoolSelect, kSlotCompact, kSlotCount };
+            kSlotPoolSelect, kSlotCompact, kSlotGramStats, kSlotCount };
+enum { kScorePhaseStats = 1, kScorePhaseColsum = 2 };
 struct Profiler;
 void prof_begin(Profiler *p, int slot, cudaStream_t st);
 void prof_end(Profiler *p, cudaStream_t st);
@@ -79,8 +80,8 @@ cudaError_t launch_gram_tc(const Plan &p, const void *dK, const UnitAddr &addr, 
 cudaError_t launch_eigen_entropy(const Plan &p, const void *d_partials, const uncomp_entropy_params &ep,
                                  float *d_entropy, float *d_erank, double *d_spectrum, uint32_t *d_status,
                                  cudaStream_t st);
-cudaError_t launch_eigen_f32(const Plan &p, const void *d_partials, const uncomp_entropy_params &ep, float *d_entropy,
-                             float *d_erank, double *d_spectrum, uint32_t *d_status, cudaStream_t st);
+cudaError_t launch_eigen_f32(const Plan &p, const void *d_partials, int partials_per_unit, const uncomp_entropy_params &ep,
+                             float *d_entropy, float *d_erank, double *d_spectrum, uint32_t *d_status, cudaStream_t st);
 cudaError_t launch_gram_reduce(const Plan &p, const void *d_partials, double *d_out, cudaStream_t st);
 int check_budget_params(const uncomp_shape &s, const uncomp_budget_params &bp);
 cudaError_t launch_budgets(const Plan &p, const float *d_erank, const uncomp_budget_params &bp, int32_t *d_budgets,
@@ -88,9 +89,11 @@ cudaError_t launch_budgets(const Plan &p, const float *d_erank, const uncomp_bud
                            int64_t *d_rem, cudaStream_t st);
 cudaError_t launch_scores_simt(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
                                float *d_stats_part, float *d_stats, float *d_raw, Profiler *prof, cudaStream_t st);
+// phases: kScorePhaseStats (pass A; with d_gram_part != NULL the Gram partials of every (unit, scorer chunk) are
+// produced in the same sweep) and / or kScorePhaseColsum (merge + pass B)
 cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
-                             float *d_stats_part, float *d_stats, float *d_raw, uint32_t *d_status, Profiler *prof,
-                             cudaStream_t st);
+                             float *d_stats_part, float *d_stats, float *d_raw, float *d_gram_part, int phases,
+                             uint32_t *d_status, Profiler *prof, cudaStream_t st);
 cudaError_t launch_pool_select(const Plan &p, const float *d_raw, float *d_pooled, int pool_kernel, int pool_mode,
                                const int32_t *d_budgets, const int64_t *d_offsets, int32_t *d_indices,
                                uint32_t *d_status, cudaStream_t st);

@@ -303,9 +303,9 @@ eigen_f32_kernel(const float *__restrict__ partials, int P, int N, int k_trunc, 
     if (spectrum && tid < k) spectrum[(size_t)u * k + tid] = S.lam[tid] * trace;
 }
 
-cudaError_t launch_eigen_f32(const Plan &p, const void *d_partials, const uncomp_entropy_params &ep, float *d_entropy,
-                             float *d_erank, double *d_spectrum, uint32_t *d_status, cudaStream_t st) {
-    eigen_f32_kernel<<<p.units, kT, 0, st>>>((const float *)d_partials, p.gram_splits, p.shape.N, ep.k_trunc, ep.center,
+cudaError_t launch_eigen_f32(const Plan &p, const void *d_partials, int partials_per_unit, const uncomp_entropy_params &ep,
+                             float *d_entropy, float *d_erank, double *d_spectrum, uint32_t *d_status, cudaStream_t st) {
+    eigen_f32_kernel<<<p.units, kT, 0, st>>>((const float *)d_partials, partials_per_unit, p.shape.N, ep.k_trunc, ep.center,
                                              ep.norm, ep.max_iters, d_entropy, d_erank, d_spectrum, d_status);
     return cudaGetLastError();
 }

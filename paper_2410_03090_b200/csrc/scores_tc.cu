@@ -16,6 +16,10 @@
 // accumulator, the other keeps the exponential unit busy); inside a group warp % 4 selects the TMEM lane
 // quarter and bit 2 of the warp index the 64-column half of an accumulator.  Warp 16 is the TMA producer,
 // warp 17 allocates TMEM and issues the MMAs.  Each group owns two of the four 128-column accumulators.
+// Mode 2 of the kernel is pass A with the Gram stage folded in: the K tile that is in shared memory for
+// Qw K^T is also the MN-major operand of G += K_tile^T K_tile (and of the narrow all-ones MMA for the column
+// sums), so the entropy stage costs no second sweep over K.  The tensor pipe has the room (pass A is bound
+// by the exponential unit); TMEM then holds one accumulator per softmax group plus the Gram block.
 // Every wait is bounded; a timeout raises UNCOMP_STATUS_TIMEOUT and the CTA drains and exits.
 #include "tc_common.cuh"
 
@@ -31,13 +35,13 @@ constexpr int kScoreThreads = kSoftThreads + 64;
 constexpr int kMaxStages = 4;
 
 struct ScoreTail {
-    uint64_t full[kMaxStages], empty[kMaxStages], qfull, tfull[kNB], tempty[kNB];
+    uint64_t full[kMaxStages], empty[kMaxStages], qfull, tfull[kNB], tempty[kNB], gfull;
     uint32_t tmem_base;
 };
 
 __host__ __device__ constexpr int score_stages(int MB) { return MB <= 2 ? 4 : (MB == 3 ? 3 : 2); }
 __host__ __device__ constexpr int score_smem(int MB) {
-    return 1024 + MB * kBlockBytes + score_stages(MB) * kBlockBytes + MB * 128 * 4 + 2 * 4 * 128 * 4 +
+    return 1024 + MB * kBlockBytes + score_stages(MB) * kBlockBytes + MB * 128 * 4 + 2 * 4 * 128 * 4 + 2048 +
            (int)sizeof(ScoreTail);
 }
 
@@ -100,11 +104,15 @@ __device__ __forceinline__ float colsum_partial(const uint32_t (&v)[64], float c
 }
 }  // namespace
 
-template <int MB, bool PASS_B>
+template <int MB, int MODE>   // MODE 0: pass A, 1: pass B, 2: pass A fused with the Gram stage
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant__ CUtensorMap tmapK, int L, int H,
                 int N, int w, int rows, int chunk, int splits, float c_log2, float *__restrict__ stats_part,
-                const float *__restrict__ mprime, float *__restrict__ raw, uint32_t *__restrict__ status) {
+                const float *__restrict__ mprime, float *__restrict__ raw, float *__restrict__ gram_part,
+                uint32_t *__restrict__ status) {
+    constexpr bool PASS_B = MODE == 1, GRAM = MODE == 2;
+    constexpr int NA = GRAM ? 1 : 2;                 // accumulators per softmax group
+    constexpr uint32_t kGramCol = 256, kSumCol = 384;  // TMEM columns of the Gram block and the column sums
     constexpr int S = score_stages(MB);
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = tc::smem_u32(smem_raw);
@@ -114,7 +122,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
     const uint32_t k_addr = q_addr + MB * kBlockBytes;
     float *mp = reinterpret_cast<float *>(smem + (MB + S) * kBlockBytes);      // [MB * 128]
     float *colsum = mp + MB * 128;                                             // [2][4][128]
-    ScoreTail &T = *reinterpret_cast<ScoreTail *>(colsum + 2 * 4 * 128);
+    unsigned char *ones = reinterpret_cast<unsigned char *>(colsum + 2 * 4 * 128);   // 2 KB, mode 2 only
+    ScoreTail &T = *reinterpret_cast<ScoreTail *>(ones + 2048);
 
     const int c = blockIdx.x, u = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -131,11 +140,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
             tc::mbar_init(tc::smem_u32(&T.empty[s]), 1);
         }
         tc::mbar_init(tc::smem_u32(&T.qfull), 1);
+        tc::mbar_init(tc::smem_u32(&T.gfull), 1);
         for (int i = 0; i < kNB; ++i) {
             tc::mbar_init(tc::smem_u32(&T.tfull[i]), 1);
             tc::mbar_init(tc::smem_u32(&T.tempty[i]), kSoftThreads / 64);   // the 8 warps of one group
         }
         tc::fence_mbar_init();
+    }
+    if (GRAM) {   // all-ones bf16 operand of the column-sum MMA
+        for (int i = threadIdx.x; i < 2048 / 4; i += kScoreThreads) reinterpret_cast<uint32_t *>(ones)[i] = 0x3f803f80u;
+        tc::fence_proxy_async();
     }
     if (warp == 17) {
         tc::tmem_alloc(tc::smem_u32(&T.tmem_base), 512);
@@ -190,6 +204,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) q_lo[mb] = tc::desc_lo(d0) + (uint32_t)(mb * kBlockBytes >> 4);
             const uint32_t k_lo0 = tc::desc_lo(tc::smem_desc_sw128(k_addr, 16, 1024));
+            const uint64_t gd = tc::smem_desc_sw128(k_addr, kHalfBytes, 1024);
+            const uint64_t od = tc::smem_desc_sw128(tc::smem_u32(ones), 1024, 1024);
+            const uint32_t g_lo0 = tc::desc_lo(gd), g_hi = tc::desc_hi(gd), ones_lo = tc::desc_lo(od), ones_hi = tc::desc_hi(od);
             bool ok = tc::mbar_wait(tc::smem_u32(&T.qfull), 0, status);
             for (int i = 0; i < ntiles && ok; ++i) {
                 const int s = i % S;
@@ -198,9 +215,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                 const uint32_t k_lo = k_lo0 + (uint32_t)(s * (kBlockBytes >> 4));
 #pragma unroll
                 for (int mb = 0; mb < MB; ++mb) {
-                    // each softmax group owns two accumulators: tile i belongs to group i & 1
-                    const int lq = (i >> 1) * MB + mb, buf = 2 * (i & 1) + (lq & 1);
-                    if (ok && lq >= 2) ok = tc::mbar_wait(tc::smem_u32(&T.tempty[buf]), ((lq >> 1) - 1) & 1, status);
+                    // tile i belongs to softmax group i & 1, which owns NA accumulators of 128 columns
+                    const int lq = (i >> 1) * MB + mb, buf = NA * (i & 1) + (lq % NA);
+                    if (ok && lq >= NA) ok = tc::mbar_wait(tc::smem_u32(&T.tempty[buf]), ((lq / NA) - 1) & 1, status);
                     if (!ok) break;
                     tc::tc_fence_after();
                     const uint32_t d_tmem = tmem + buf * 128;
@@ -212,8 +229,22 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                     }
                     tc::mma_commit(tc::smem_u32(&T.tfull[buf]));
                 }
+                if (GRAM && ok) {
+                    // G += K_tile^T K_tile, s += K_tile^T 1: the same stage read MN-major (feature halves
+                    // kHalfBytes apart, 8-token groups 1024 B apart); 16 tokens further = +128 address units
+                    constexpr uint32_t idesc_g = tc::idesc_bf16_f32(128, 128, 1, 1);
+                    constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, 16, 1, 1);
+                    const uint32_t g_lo = g_lo0 + (uint32_t)(s * (kBlockBytes >> 4));
+#pragma unroll
+                    for (int k = 0; k < kTile / 16; ++k) {
+                        const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
+                        tc::mma_f16_ss_lohi(tmem + kGramCol, g_lo + k * 128, g_lo + k * 128, g_hi, idesc_g, acc);
+                        tc::mma_f16_ss2(tmem + kSumCol, g_lo + k * 128, g_hi, ones_lo, ones_hi, idesc_s, acc);
+                    }
+                }
                 tc::mma_commit(tc::smem_u32(&T.empty[s]));
             }
+            if (GRAM) tc::mma_commit(tc::smem_u32(&T.gfull));
         }
     } else {
         // ---------------- softmax warps ----------------
@@ -236,10 +267,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
             float acc = 0.f;
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
-                const int lq = (i >> 1) * MB + mb, buf = 2 * group + (lq & 1);
+                const int lq = (i >> 1) * MB + mb, buf = NA * group + (lq % NA);
                 uint32_t v[64];
                 if (!dead) {
-                    const bool ok = tc::mbar_wait(tc::smem_u32(&T.tfull[buf]), (lq >> 1) & 1, status);
+                    const bool ok = tc::mbar_wait(tc::smem_u32(&T.tfull[buf]), (lq / NA) & 1, status);
                     dead = !__all_sync(0xffffffffu, ok);
                 }
                 if (!dead) {
@@ -304,6 +335,29 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                 }
             }
         }
+        if (GRAM) {
+            // drain the Gram block: warp (quarter, cb) stores rows 32 quarter .. +31, columns 32 cb .. +31
+            bool ok = ntiles > 0 && tc::mbar_wait(tc::smem_u32(&T.gfull), 0, status);
+            ok = __all_sync(0xffffffffu, ok) && !dead;
+            if (ok) {
+                tc::tc_fence_after();
+                const int cb = warp >> 2;
+                float *out = gram_part + ((size_t)u * splits + c) * (kD * kD + kD);
+                uint32_t r[32];
+                tc::tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + kGramCol + cb * 32, r);
+                tc::tmem_ld_wait();
+                float4 *dst = reinterpret_cast<float4 *>(out + (size_t)lane_row * kD + cb * 32);
+#pragma unroll
+                for (int q4 = 0; q4 < 8; ++q4)
+                    dst[q4] = make_float4(__uint_as_float(r[4 * q4]), __uint_as_float(r[4 * q4 + 1]),
+                                          __uint_as_float(r[4 * q4 + 2]), __uint_as_float(r[4 * q4 + 3]));
+                if (cb == 0) {
+                    tc::tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + kSumCol, r);   // only column 0 is used
+                    tc::tmem_ld_wait();
+                    out[kD * kD + lane_row] = __uint_as_float(r[0]);
+                }
+            }
+        }
     }
     tc::tc_fence_before();
     __syncthreads();
@@ -328,41 +382,46 @@ __global__ void score_tc_merge_kernel(const float *__restrict__ stats_part, int 
 
 template <int MB>
 static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, const CUtensorMap &tk, float c_log2,
-                                       float *d_stats_part, float *d_mprime, float *d_raw, uint32_t *d_status,
-                                       Profiler *prof, cudaStream_t st) {
+                                       float *d_stats_part, float *d_mprime, float *d_raw, float *d_gram_part,
+                                       int phases, uint32_t *d_status, Profiler *prof, cudaStream_t st) {
     const uncomp_shape &s = p.shape;
     const int smem = score_smem(MB);
-    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<MB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<MB, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(score_tc_kernel<MB, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(score_tc_kernel<MB, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(score_tc_kernel<MB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    {
-        ProfScope ps(prof, kSlotScoreStats, st);
+    if (phases & kScorePhaseStats) {
+        ProfScope ps(prof, d_gram_part ? kSlotGramStats : kSlotScoreStats, st);
         dim3 grid(p.score_splits, p.units);
-        score_tc_kernel<MB, false><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
+        if (d_gram_part)
+            score_tc_kernel<MB, 2><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
                                                                       p.score_splits, c_log2, d_stats_part, nullptr,
-                                                                      nullptr, d_status);
+                                                                      nullptr, d_gram_part, d_status);
+        else
+            score_tc_kernel<MB, 0><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
+                                                                      p.score_splits, c_log2, d_stats_part, nullptr,
+                                                                      nullptr, nullptr, d_status);
     }
-    {
-        ProfScope ps(prof, kSlotStatsMerge, st);
-        const int total = p.units * p.rows;
-        score_tc_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows, p.score_splits,
-                                                                   d_mprime);
-    }
-    {
+    if (phases & kScorePhaseColsum) {
+        {
+            ProfScope ps(prof, kSlotStatsMerge, st);
+            const int total = p.units * p.rows;
+            score_tc_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows, p.score_splits,
+                                                                       d_mprime);
+        }
         ProfScope ps(prof, kSlotScoreColsum, st);
         const int splitsB = (p.prefix + p.score_chunk - 1) / p.score_chunk;
         dim3 grid(splitsB, p.units);
-        score_tc_kernel<MB, true><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
-                                                                     splitsB, c_log2, nullptr, d_mprime, d_raw,
-                                                                     d_status);
+        score_tc_kernel<MB, 1><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
+                                                                  splitsB, c_log2, nullptr, d_mprime, d_raw, nullptr,
+                                                                  d_status);
     }
     return cudaGetLastError();
 }
 
 cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
-                             float *d_stats_part, float *d_stats, float *d_raw, uint32_t *d_status, Profiler *prof,
-                             cudaStream_t st) {
+                             float *d_stats_part, float *d_stats, float *d_raw, float *d_gram_part, int phases,
+                             uint32_t *d_status, Profiler *prof, cudaStream_t st) {
     CUtensorMap tq, tk;
     cudaError_t e = make_query_tensor_map(&tq, dQw, p.units, p.rows);
     if (e != cudaSuccess) return e;
@@ -371,10 +430,10 @@ cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, con
     const float c_log2 = scale * 1.4426950408889634f;
     const int MB = (p.rows + 127) / 128;
     switch (MB) {
-        case 1: return launch_scores_tc_mb<1>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_status, prof, st);
-        case 2: return launch_scores_tc_mb<2>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_status, prof, st);
-        case 3: return launch_scores_tc_mb<3>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_status, prof, st);
-        default: return launch_scores_tc_mb<4>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_status, prof, st);
+        case 1: return launch_scores_tc_mb<1>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        case 2: return launch_scores_tc_mb<2>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        case 3: return launch_scores_tc_mb<3>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        default: return launch_scores_tc_mb<4>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
     }
 }
 

@@ -331,3 +331,43 @@ def test_bf16_spectrum_register_kernel_vs_oracle():
         got = spec.reshape(-1, 128)[u].cpu().numpy()
         np.testing.assert_allclose(got, lam, rtol=0, atol=2e-6 * lam[0])
         assert abs(float(ent.reshape(-1)[u]) - H) <= 1e-4 * max(abs(H), 1.0)
+
+
+def test_fused_entropy_statistics_sweep_matches_separate_calls():
+    # uncomp_entropy with the window queries forms the Gram matrices and the scorer's row statistics in one
+    # sweep over K; everything downstream must agree with the two-sweep path
+    from paper_2410_03090_b200.compress import CompressionPass
+    wl = synth.scaled(synth.WORKLOADS["c3"], N=9001, L=2)          # two scorer chunks, ragged tail
+    K, V, Qw = synth.generate(wl, "cuda")
+    outs = []
+    for fused in (True, False):
+        cp = CompressionPass(wl, "cuda", fused=fused)
+        o = cp.run(K, V, Qw)
+        torch.cuda.synchronize()
+        assert cp.status() == 0
+        outs.append({k: getattr(o, k).clone() for k in ("entropy", "budgets", "scores", "indices", "Kc", "Vc")})
+    f, u = outs
+    assert float((f["entropy"] - u["entropy"]).abs().max()) < 2e-6
+    assert torch.equal(f["scores"], u["scores"])                   # same statistics, bit for bit
+    if torch.equal(f["budgets"], u["budgets"]):
+        assert torch.equal(f["indices"], u["indices"]) and torch.equal(f["Kc"], u["Kc"]) and torch.equal(f["Vc"], u["Vc"])
+    _check_all(wl, K, V, Qw, CompressionPass(wl, "cuda", fused=True).run(K, V, Qw), range(0, wl.units, 5))
+
+
+def test_fused_gram_is_exact_on_integer_keys():
+    # integer-valued keys: every Gram partial is exact in fp32 whatever the chunking, so the fused sweep and the
+    # stand-alone Gram kernel (itself pinned against the oracle exactly) must give identical spectra
+    ub = _ub()
+    N, H, G, w = 8192 + 300, 4, 2, 16
+    g = torch.Generator(device="cuda").manual_seed(11)
+    K = torch.randint(-3, 4, (1, 1, H, N, 128), generator=g, device="cuda").to(torch.bfloat16)
+    Qw = torch.randn(1, 1, H * G, w, 128, generator=g, device="cuda").to(torch.bfloat16)
+    ctx = ub.Context(ub.make_shape(1, 1, H, H * G, N, 128, w, "bf16"))
+    spec_f = torch.empty(1, 1, H, 128, dtype=torch.float64, device="cuda")
+    spec_u = torch.empty_like(spec_f)
+    ent_f, _ = ub.uncomp_entropy(ctx, K, k_trunc=128, spectrum=spec_f, Qw=Qw)
+    ent_f = ent_f.clone()
+    ent_u, _ = ub.uncomp_entropy(ctx, K, k_trunc=128, spectrum=spec_u)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    assert torch.equal(spec_f, spec_u) and torch.equal(ent_f, ent_u)
