@@ -39,16 +39,18 @@ struct E32Smem {
     int flags[2];
 };
 
-__device__ __forceinline__ int sturm_count_n(const double *dn, const double *e2, double x) {
+// Number of eigenvalues of the normalised tridiagonal matrix that are < x: sign changes of the three-term
+// recurrence p_i = (d_i - x) p_{i-1} - e_{i-1}^2 p_{i-2}.  Robust form: a zero takes the sign opposite to
+// its predecessor and the pair is rescaled whenever it gets small.
+__device__ __noinline__ int sturm_count_robust(const double *dn, const double *e2, double x) {
     const double tiny = 0x1p-400, big = 0x1p+400;
     double p0 = 0.0, p1 = 1.0;
     bool neg1 = false;
     int count = 0;
-#pragma unroll 4
     for (int i = 0; i < n; ++i) {
         double pn = (dn[i] - x) * p1 - e2[i] * p0;
         bool negn = pn < 0.0;
-        if (pn == 0.0) {            // a zero takes the sign opposite to its predecessor
+        if (pn == 0.0) {
             negn = !neg1;
             pn = (negn ? -1.0 : 1.0) * fabs(p1) * 0x1p-100;
         }
@@ -58,6 +60,35 @@ __device__ __forceinline__ int sturm_count_n(const double *dn, const double *e2,
         neg1 = negn;
         if (fabs(p1) < tiny) { p1 *= big; p0 *= big; }
     }
+    return count;
+}
+
+// Fast form of the same count: one dependent fused multiply-add per step, signs compared on the raw bit
+// patterns, the magnitude checked (and an exact zero looked for) only every 8 steps.  With |d_i - x| <= 2 and
+// e^2 <= 1 the pair grows by at most 2^10 in 8 steps and shrinks by at most 2^-53 per step, so the window
+// [2^-400, 2^400] keeps it far from overflow and underflow.  An exact zero (x hits an eigenvalue of a
+// leading block bit for bit) is rare; the robust form then recounts.
+__device__ __forceinline__ int sturm_count_n(const double *dn, const double *e2, double x) {
+    double p0 = 1.0, p1 = dn[0] - x;
+    int count = __double2hiint(p1) < 0 ? 1 : 0;      // sign change against p_0 = 1
+    bool zero = p1 == 0.0;
+#pragma unroll 1
+    for (int i0 = 1; i0 < n; i0 += 8) {
+#pragma unroll
+        for (int i = i0; i < i0 + 8; ++i) {
+            if (i < n) {
+                const double pn = fma(dn[i] - x, p1, -(e2[i] * p0));
+                count += (unsigned)(__double2hiint(pn) ^ __double2hiint(p1)) >> 31;
+                zero |= pn == 0.0;
+                p0 = p1;
+                p1 = pn;
+            }
+        }
+        const double a = fabs(p1);
+        if (a < 0x1p-400) { p1 *= 0x1p+400; p0 *= 0x1p+400; }
+        else if (a > 0x1p+400) { p1 *= 0x1p-400; p0 *= 0x1p-400; }
+    }
+    if (zero) return sturm_count_robust(dn, e2, x);
     return count;
 }
 
@@ -244,7 +275,7 @@ eigen_f32_kernel(const float *__restrict__ partials, int P, int N, int k_trunc, 
 
     const int k = min(k_trunc, n);
     const int iters = max_iters > 0 ? max_iters : 10;
-    const double tol = 1e-8;
+    const double tol = 2e-8;    // of the spectral radius; the fp32 reduction itself is good to about 1e-7
     const int sub = tid & 7;
     const unsigned team_mask = 0xffu << (lane & 24);
     for (int j0 = 0; j0 < k; j0 += kT / 8) {
