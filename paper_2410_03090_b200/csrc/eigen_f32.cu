@@ -31,6 +31,8 @@ struct E32Smem {
     double e2[n];      // (off-diagonal / scale)^2, e2[0] = 0
     double lam[n];
     double red[8];
+    float dnf[n];      // fp32 copies for the fast Sturm count
+    float e2f[n];
     float xs[n];
     float ps[n];
     float dd[n];
@@ -63,32 +65,34 @@ __device__ __noinline__ int sturm_count_robust(const double *dn, const double *e
     return count;
 }
 
-// Fast form of the same count: one dependent fused multiply-add per step, signs compared on the raw bit
-// patterns, the magnitude checked (and an exact zero looked for) only every 8 steps.  With |d_i - x| <= 2 and
-// e^2 <= 1 the pair grows by at most 2^10 in 8 steps and shrinks by at most 2^-53 per step, so the window
-// [2^-400, 2^400] keeps it far from overflow and underflow.  An exact zero (x hits an eigenvalue of a
-// leading block bit for bit) is rare; the robust form then recounts.
-__device__ __forceinline__ int sturm_count_n(const double *dn, const double *e2, double x) {
-    double p0 = 1.0, p1 = dn[0] - x;
-    int count = __double2hiint(p1) < 0 ? 1 : 0;      // sign change against p_0 = 1
-    bool zero = p1 == 0.0;
+// Fast form of the same count in fp32 (the tridiagonal matrix comes from an fp32 reduction, so its entries
+// carry no more than fp32 accuracy anyway): one dependent fused multiply-add per step, signs compared on
+// the raw bit patterns, the magnitude checked (and an exact zero looked for) every 4 steps.  With
+// |d_i - x| <= 2 and e^2 <= 1 the pair grows by at most 2^6 in 4 steps and one step shrinks it by at most
+// 2^-24, so re-centring into [2^-20, 2^20] every 4 steps keeps it inside the fp32 range.  An exact zero is
+// rare; the robust fp64 form then recounts.
+__device__ __forceinline__ int sturm_count_n(const double *dn, const double *e2, const float *dnf, const float *e2f,
+                                             float x) {
+    float p0 = 1.f, p1 = dnf[0] - x;
+    int count = __float_as_int(p1) < 0 ? 1 : 0;      // sign change against p_0 = 1
+    bool zero = p1 == 0.f;
 #pragma unroll 1
-    for (int i0 = 1; i0 < n; i0 += 8) {
+    for (int i0 = 1; i0 < n; i0 += 4) {
 #pragma unroll
-        for (int i = i0; i < i0 + 8; ++i) {
+        for (int i = i0; i < i0 + 4; ++i) {
             if (i < n) {
-                const double pn = fma(dn[i] - x, p1, -(e2[i] * p0));
-                count += (unsigned)(__double2hiint(pn) ^ __double2hiint(p1)) >> 31;
-                zero |= pn == 0.0;
+                const float pn = fmaf(dnf[i] - x, p1, -(e2f[i] * p0));
+                count += (unsigned)(__float_as_int(pn) ^ __float_as_int(p1)) >> 31;
+                zero |= pn == 0.f;
                 p0 = p1;
                 p1 = pn;
             }
         }
-        const double a = fabs(p1);
-        if (a < 0x1p-400) { p1 *= 0x1p+400; p0 *= 0x1p+400; }
-        else if (a > 0x1p+400) { p1 *= 0x1p-400; p0 *= 0x1p-400; }
+        const float a = fabsf(p1);
+        if (a < 0x1p-20f) { p1 *= 0x1p+40f; p0 *= 0x1p+40f; }
+        else if (a > 0x1p+20f) { p1 *= 0x1p-40f; p0 *= 0x1p-40f; }
     }
-    if (zero) return sturm_count_robust(dn, e2, x);
+    if (zero) return sturm_count_robust(dn, e2, (double)x);
     return count;
 }
 
@@ -221,17 +225,35 @@ eigen_f32_kernel(const float *__restrict__ partials, int P, int N, int k_trunc, 
     __syncthreads();
     const double trace = S.red[0] + S.red[1] + S.red[2] + S.red[3];
     const double inv_tr = trace > 0.0 ? 1.0 / trace : 0.0;
+    // Coalesced 16-byte loads of the partials (many in flight), summed and centred in fp64, scaled to unit
+    // trace and staged in shared memory; each thread then picks its 64 entries from there.
+    extern __shared__ __align__(16) float stage[];        // [n * n]
+    {
+        const float4 *base4 = reinterpret_cast<const float4 *>(base);
+        constexpr int len4 = len / 4;
+#pragma unroll 4
+        for (int i = 0; i < n * n / 4 / kT; ++i) {
+            const int e4 = tid + kT * i;
+            double g0 = 0.0, g1 = 0.0, g2 = 0.0, g3 = 0.0;
+            for (int p = 0; p < P; ++p) {
+                const float4 v = __ldg(base4 + (size_t)p * len4 + e4);
+                g0 += (double)v.x; g1 += (double)v.y; g2 += (double)v.z; g3 += (double)v.w;
+            }
+            const int r = (4 * e4) >> 7, c0 = (4 * e4) & 127;
+            if (center) {
+                const double sr = S.sd[r] * invN;
+                g0 -= sr * S.sd[c0]; g1 -= sr * S.sd[c0 + 1]; g2 -= sr * S.sd[c0 + 2]; g3 -= sr * S.sd[c0 + 3];
+            }
+            *reinterpret_cast<float4 *>(stage + 4 * e4) =
+                make_float4((float)(g0 * inv_tr), (float)(g1 * inv_tr), (float)(g2 * inv_tr), (float)(g3 * inv_tr));
+        }
+    }
+    __syncthreads();
     float A[8][8];
 #pragma unroll
     for (int a = 0; a < 8; ++a)
 #pragma unroll
-        for (int b = 0; b < 8; ++b) {
-            const int r = ty + 16 * a, c = tx + 16 * b;
-            double g = 0.0;
-            for (int p = 0; p < P; ++p) g += (double)base[(size_t)p * len + r * n + c];
-            if (center) g -= S.sd[r] * S.sd[c] * invN;
-            A[a][b] = (float)(g * inv_tr);
-        }
+        for (int b = 0; b < 8; ++b) A[a][b] = stage[(ty + 16 * a) * n + tx + 16 * b];
 
     // ---- 2. Householder tridiagonalisation in registers -----------------------------------------
     householder_block<0>(A, S, tx, ty, tid);
@@ -265,11 +287,13 @@ eigen_f32_kernel(const float *__restrict__ partials, int P, int N, int k_trunc, 
         S.dn[tid] = (double)S.dd[tid] * inv_scale;
         const double e = tid > 0 ? (double)S.ee[tid - 1] * inv_scale : 0.0;
         S.e2[tid] = e * e;
+        S.dnf[tid] = (float)S.dn[tid];
+        S.e2f[tid] = (float)(e * e);
     }
     __syncthreads();
     // coarse round: counts at 256 interior points of [lo0, hi0], shared by all eigenvalues
     const double lo0 = -1.0, hi0 = 1.0 + 0x1p-40, step0 = (hi0 - lo0) / (double)(kT + 1);
-    S.cnt[tid + 1] = sturm_count_n(S.dn, S.e2, lo0 + step0 * (double)(tid + 1));
+    S.cnt[tid + 1] = sturm_count_n(S.dn, S.e2, S.dnf, S.e2f, (float)(lo0 + step0 * (double)(tid + 1)));
     if (tid == 0) { S.cnt[0] = 0; S.cnt[kT + 1] = n; }
     __syncthreads();
 
@@ -298,7 +322,7 @@ eigen_f32_kernel(const float *__restrict__ partials, int P, int N, int k_trunc, 
             const bool done = width <= tol;
             if (__all_sync(0xffffffffu, done)) break;
             int c = 0;
-            if (!done) c = sturm_count_n(S.dn, S.e2, lo + width * (double)(sub + 1) * (1.0 / 9.0));
+            if (!done) c = sturm_count_n(S.dn, S.e2, S.dnf, S.e2f, (float)(lo + width * (double)(sub + 1) * (1.0 / 9.0)));
             const unsigned above = __ballot_sync(0xffffffffu, c > idx) & team_mask;
             if (!done) {
                 const int f = above ? (__ffs(above) - 1) - (lane & 24) : 8;
@@ -336,7 +360,10 @@ eigen_f32_kernel(const float *__restrict__ partials, int P, int N, int k_trunc, 
 
 cudaError_t launch_eigen_f32(const Plan &p, const void *d_partials, int partials_per_unit, const uncomp_entropy_params &ep,
                              float *d_entropy, float *d_erank, double *d_spectrum, uint32_t *d_status, cudaStream_t st) {
-    eigen_f32_kernel<<<p.units, kT, 0, st>>>((const float *)d_partials, partials_per_unit, p.shape.N, ep.k_trunc, ep.center,
+    const int smem = n * n * (int)sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(eigen_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    eigen_f32_kernel<<<p.units, kT, smem, st>>>((const float *)d_partials, partials_per_unit, p.shape.N, ep.k_trunc, ep.center,
                                              ep.norm, ep.max_iters, d_entropy, d_erank, d_spectrum, d_status);
     return cudaGetLastError();
 }
