@@ -24,6 +24,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+EXP_KERNELS = ("score_stats", "score_colsum", "gram_score_stats")
 METRIC = "compression_pass_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -282,6 +283,12 @@ def main():
         if work is not None:
             ach = work / (avg_ms / 1e3)
             ent.update({"achieved": round(ach, 2), "peak": peak, "unit": unit, "frac": round(ach / peak, 4)})
+        if name in EXP_KERNELS:
+            # second ceiling of the scorer kernels: the exponential unit, 16 ex2 per clock per SM
+            n_exp = wl.units * wl.G * wl.w * (wl.N if name != "score_colsum" else wl.N - wl.w)
+            sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+            peak_exp = sm_count * 16 * (clocks.get("sm_max_mhz") or 1965) * 1e6
+            ent.update({"ex2_per_launch": n_exp, "ex2_frac_of_unit_peak": round(n_exp / (avg_ms / 1e3) / peak_exp, 4)})
         kernels[name] = ent
     total_kernel_ms = sum(v[0] for v in prof.values())
     for name in kernels:

@@ -207,6 +207,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
             const uint64_t gd = tc::smem_desc_sw128(k_addr, kHalfBytes, 1024);
             const uint64_t od = tc::smem_desc_sw128(tc::smem_u32(ones), 1024, 1024);
             const uint32_t g_lo0 = tc::desc_lo(gd), g_hi = tc::desc_hi(gd), ones_lo = tc::desc_lo(od), ones_hi = tc::desc_hi(od);
+            // Mode 2: the Gram MMAs of a tile only have to be issued before its stage is handed back, so they
+            // are deferred by up to one tile and issued while this thread would otherwise wait for an
+            // accumulator: the latency-critical QK^T MMAs never queue behind them.
+            int g_done = 0;                    // tiles whose Gram MMAs are issued (and whose stage is released)
+            auto issue_gram = [&](int t) {
+                constexpr uint32_t idesc_g = tc::idesc_bf16_f32(128, 128, 1, 1);
+                constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, 16, 1, 1);
+                const int sg = t % S;
+                const uint32_t g_lo = g_lo0 + (uint32_t)(sg * (kBlockBytes >> 4));
+#pragma unroll
+                for (int k = 0; k < kTile / 16; ++k) {
+                    // the same stage read MN-major (feature halves kHalfBytes apart, 8-token groups 1024 B
+                    // apart); 16 tokens further = +128 address units
+                    const uint32_t acc = (t > 0 || k > 0) ? 1u : 0u;
+                    tc::mma_f16_ss_lohi(tmem + kGramCol, g_lo + k * 128, g_lo + k * 128, g_hi, idesc_g, acc);
+                    tc::mma_f16_ss2(tmem + kSumCol, g_lo + k * 128, g_hi, ones_lo, ones_hi, idesc_s, acc);
+                }
+                tc::mma_commit(tc::smem_u32(&T.empty[sg]));
+            };
             bool ok = tc::mbar_wait(tc::smem_u32(&T.qfull), 0, status);
             for (int i = 0; i < ntiles && ok; ++i) {
                 const int s = i % S;
@@ -217,7 +236,23 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                 for (int mb = 0; mb < MB; ++mb) {
                     // tile i belongs to softmax group i & 1, which owns NA accumulators of 128 columns
                     const int lq = (i >> 1) * MB + mb, buf = NA * (i & 1) + (lq % NA);
-                    if (ok && lq >= NA) ok = tc::mbar_wait(tc::smem_u32(&T.tempty[buf]), ((lq / NA) - 1) & 1, status);
+                    if (ok && lq >= NA) {
+                        const uint32_t bar = tc::smem_u32(&T.tempty[buf]);
+                        const uint32_t parity = ((lq / NA) - 1) & 1;
+                        if (GRAM) {
+                            uint32_t spins = 0;
+                            while (!tc::mbar_try_wait(bar, parity)) {
+                                if (g_done < i) issue_gram(g_done++);
+                                else if (++spins >= tc::kSpinLimit) {
+                                    atomicOr(status, (uint32_t)UNCOMP_STATUS_TIMEOUT);
+                                    ok = false;
+                                    break;
+                                }
+                            }
+                        } else {
+                            ok = tc::mbar_wait(bar, parity, status);
+                        }
+                    }
                     if (!ok) break;
                     tc::tc_fence_after();
                     const uint32_t d_tmem = tmem + buf * 128;
@@ -229,22 +264,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                     }
                     tc::mma_commit(tc::smem_u32(&T.tfull[buf]));
                 }
-                if (GRAM && ok) {
-                    // G += K_tile^T K_tile, s += K_tile^T 1: the same stage read MN-major (feature halves
-                    // kHalfBytes apart, 8-token groups 1024 B apart); 16 tokens further = +128 address units
-                    constexpr uint32_t idesc_g = tc::idesc_bf16_f32(128, 128, 1, 1);
-                    constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, 16, 1, 1);
-                    const uint32_t g_lo = g_lo0 + (uint32_t)(s * (kBlockBytes >> 4));
-#pragma unroll
-                    for (int k = 0; k < kTile / 16; ++k) {
-                        const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
-                        tc::mma_f16_ss_lohi(tmem + kGramCol, g_lo + k * 128, g_lo + k * 128, g_hi, idesc_g, acc);
-                        tc::mma_f16_ss2(tmem + kSumCol, g_lo + k * 128, g_hi, ones_lo, ones_hi, idesc_s, acc);
-                    }
+                if (!ok) break;
+                if (GRAM) {
+                    while (g_done < i) issue_gram(g_done++);      // at most one tile may stay pending
+                } else {
+                    tc::mma_commit(tc::smem_u32(&T.empty[s]));
                 }
-                tc::mma_commit(tc::smem_u32(&T.empty[s]));
             }
-            if (GRAM) tc::mma_commit(tc::smem_u32(&T.gfull));
+            if (GRAM) {
+                if (ok) while (g_done < ntiles) issue_gram(g_done++);
+                tc::mma_commit(tc::smem_u32(&T.gfull));
+            }
         }
     } else {
         // ---------------- softmax warps ----------------
@@ -308,8 +338,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
             }
         }
         if (!PASS_B) {
-            // merge the four (group, half) partials of every row in a fixed order; the K stages are idle by now
-            float2 *merge = reinterpret_cast<float2 *>(smem + MB * kBlockBytes);      // [4][MB * 128]
+            // merge the four (group, half) partials of every row in a fixed order.  Scratch: the query blocks,
+            // which no MMA reads any more once both groups have consumed every accumulator (the K stages may still
+            // feed deferred Gram MMAs).
+            float2 *merge = reinterpret_cast<float2 *>(smem);                         // [4][MB * 128]
+            all_soft_barrier();            // both groups have consumed their last accumulator
             const int slot = group * 2 + half;
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) merge[slot * (MB * 128) + mb * 128 + lane_row] = make_float2(m_run[mb], l_run[mb]);
