@@ -24,6 +24,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes per (unit x token) of one launch, dram__bytes_read.sum + dram__bytes_write.sum from the ncu capture
+# summarised in profiles/kernels_c3_N16384_L10_ncu_full.md (80 units x 16384 tokens; traffic grows with
+# units x tokens, so a full-size launch is scaled by that product).  Set to None when a kernel changes.
+TRAFFIC_PER_UNIT_TOKEN = {"gram_score_stats": (340.92e6 + 33.37e6) / (80 * 16384),
+                          "score_colsum": (341.00e6 + 7.15e6) / (80 * 16384)}
 EXP_KERNELS = ("score_stats", "score_colsum", "gram_score_stats")
 METRIC = "compression_pass_tokens_per_s"
 UNIT = "tokens/s"
@@ -296,7 +301,10 @@ def main():
     dom = max(kernels, key=lambda n: kernels[n]["share"])
     kd = kernels[dom]
     roofline = {"kernel": dom, "bound": kd["bound"], "achieved": kd.get("achieved"), "peak": kd.get("peak"),
-                "unit": kd.get("unit"), "frac": kd.get("frac"), "traffic": None,
+                "unit": kd.get("unit"), "frac": kd.get("frac"),
+                "traffic": (round(TRAFFIC_PER_UNIT_TOKEN[dom] * wl.units * wl.N / 1e9, 4)
+                            if TRAFFIC_PER_UNIT_TOKEN.get(dom) else None),
+                "traffic_unit": "GB per launch (ncu dram bytes of a smaller case, scaled by units x tokens)",
                 "peak_source": f"of {peaks['source']} ({'sustained bf16' if kd['bound'] == 'tensor' else 'copy'})",
                 "avg_ms": kd["avg_ms"], "share": kd["share"]}
     alg_bytes = wl.algorithmic_bytes()
