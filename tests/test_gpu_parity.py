@@ -371,3 +371,36 @@ def test_fused_gram_is_exact_on_integer_keys():
     torch.cuda.synchronize()
     assert ub.uncomp_status(ctx) == 0
     assert torch.equal(spec_f, spec_u) and torch.equal(ent_f, ent_u)
+
+
+@pytest.mark.parametrize("N,w,G", [(65, 64, 4), (33, 32, 1), (130, 2, 8), (129, 1, 2)])
+def test_degenerate_lengths(N, w, G):
+    # prefix of one token, sequences shorter than / just above one 128-token tile, single-row windows
+    from dataclasses import replace
+    from paper_2410_03090_b200.compress import CompressionPass
+    base = synth.scaled(synth.WORKLOADS["c2"], N=max(N, 256), L=1)
+    P = N - w
+    avg = w + max(1, P // 2)
+    wl = replace(base, N=N, w=w, Hq=base.H * G, avg_budget=avg, n_max=avg, M=1, name=f"tiny{N}")
+    K, V, Qw = synth.generate(wl, "cuda")
+    cp = CompressionPass(wl, "cuda")
+    out = cp.run(K, V, Qw)
+    torch.cuda.synchronize()
+    assert cp.status() == 0
+    _check_all(wl, K, V, Qw, out, range(wl.units))
+
+
+def test_scores_may_stay_in_the_workspace():
+    # d_scores = NULL: the pooled scores live in the workspace; selection must be unchanged
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=900, L=1)
+    K, V, Qw = synth.generate(wl, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    er = torch.linspace(30, 2, wl.H, device="cuda").view(1, 1, wl.H).contiguous()
+    b, o, _, _ = ub.uncomp_assign_budgets(ctx, er, wl.avg_budget, wl.M, wl.n_max)
+    scores = torch.empty(wl.B, wl.L, wl.H, wl.N - wl.w, device="cuda")
+    idx_a = ub.uncomp_score_select(ctx, Qw, K, b, o, wl.total_rows, scores=scores).clone()
+    idx_b = ub.uncomp_score_select(ctx, Qw, K, b, o, wl.total_rows, scores=None)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0 and torch.equal(idx_a, idx_b)
+    parity.check_select(wl, scores, b, o, idx_b, range(wl.units))
