@@ -33,6 +33,8 @@ _lib.oracle_budgets.argtypes = [_dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int
 _lib.oracle_budgets.restype = C.c_int
 _lib.oracle_window_scores.argtypes = [_dp, _dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _dp]
 _lib.oracle_window_scores.restype = None
+_lib.oracle_last_token_scores.argtypes = [_dp, _dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _dp]
+_lib.oracle_last_token_scores.restype = None
 _lib.oracle_pool.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _dp]
 _lib.oracle_pool.restype = None
 _lib.oracle_select.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _i32p]
@@ -144,4 +146,16 @@ def compact(src_rows: np.ndarray, idx) -> np.ndarray:
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     out = np.empty((idx.shape[0], src.shape[1]), dtype=np.uint8)
     _lib.oracle_compact(_p(src, _u8p), src.shape[1], _p(idx, _i32p), idx.shape[0], _p(out, _u8p))
+    return out
+
+
+def last_token_scores(q, K, scale: float | None = None) -> np.ndarray:
+    """Hidden-state eviction scores [N] of one sequence and layer: q [Hq, d] (last position), K [H, N, d]."""
+    q, K = _f64(q), _f64(K)
+    Hq, d = q.shape
+    H, N, _ = K.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    out = np.empty(N, dtype=np.float64)
+    _lib.oracle_last_token_scores(_p(q, _dp), _p(K, _dp), H, Hq, N, d, float(scale), _p(out, _dp))
     return out

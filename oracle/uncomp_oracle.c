@@ -17,6 +17,8 @@
  *                         positions summed per key position
  *   selection             same paragraph: keep the highest-scored tokens within the head's budget; the
  *                         recent (window) tokens are part of the budget (Section 4, recent/historical split)
+ *   hidden-state eviction Section 3.3.2, "Hidden State Eviction": tokens kept for the next layer group by
+ *                         the last token's attention scores
  *   compaction            per-head ragged cache (Section 3.3.3, "each head maintains its context window");
  *                         K and V share one selection (Table 1 caption)
  *
@@ -367,4 +369,37 @@ void oracle_compact(const unsigned char *src, size_t row_bytes, const int32_t *i
 {
     for (int t = 0; t < count; ++t)
         memcpy(dst + (size_t)t * row_bytes, src + (size_t)idx[t] * row_bytes, row_bytes);
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Hidden-state eviction between layer groups (Section 3.3.2, "Hidden State Eviction"): the tokens kept
+ * for the next layer are chosen by the attention scores of the LAST token of the current layer.
+ *
+ * q is [Hq, d] (the last position's query of every query head), K is [H, N, d] (the layer's keys; query
+ * head h attends to KV head h / (Hq / H)).  Each head's logits scale * (q_h . k_j) over all N positions
+ * go through a softmax; score[j] is the sum over the Hq heads.  score has N entries.
+ * Readings (the paper gives one sentence): heads are summed, scale 1/sqrt(d) by the caller.  The caller
+ * keeps the last position unconditionally and selects among the first N - 1 (oracle_select with w = 1).
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_last_token_scores(const double *q, const double *K, int H, int Hq, int N, int d, double scale,
+                              double *score)
+{
+    const int G = Hq / H;
+    double *s = (double *)malloc((size_t)N * sizeof(double));
+    for (int j = 0; j < N; ++j) score[j] = 0.0;
+    for (int h = 0; h < Hq; ++h) {
+        const double *qh = q + (size_t)h * d;
+        const double *Kh = K + (size_t)(h / G) * N * d;
+        double mx = -INFINITY;
+        for (int j = 0; j < N; ++j) {
+            double acc = 0.0;
+            for (int a = 0; a < d; ++a) acc += qh[a] * Kh[(size_t)j * d + a];
+            s[j] = scale * acc;
+            if (s[j] > mx) mx = s[j];
+        }
+        double denom = 0.0;
+        for (int j = 0; j < N; ++j) denom += exp(s[j] - mx);
+        for (int j = 0; j < N; ++j) score[j] += exp(s[j] - mx) / denom;
+    }
+    free(s);
 }

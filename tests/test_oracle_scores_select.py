@@ -119,3 +119,50 @@ def test_compact_is_bitwise():
     idx = np.array([0, 3, 4, 19, 18], dtype=np.int32)
     out = oracle.compact(src, idx)
     assert out.tobytes() == src[idx].tobytes()
+
+
+# ------------------------------------------------------------------ hidden-state eviction scores
+def _brute_last_token(q, K, scale):
+    Hq, d = q.shape
+    H, N, _ = K.shape
+    G = Hq // H
+    out = [0.0] * N
+    for h in range(Hq):
+        lg = [scale * sum(q[h, a] * K[h // G, j, a] for a in range(d)) for j in range(N)]
+        m = max(lg)
+        ex = [math.exp(x - m) for x in lg]
+        z = sum(ex)
+        for j in range(N):
+            out[j] += ex[j] / z
+    return np.array(out)
+
+
+@pytest.mark.parametrize("H,Hq,N,d", [(2, 4, 19, 6), (1, 1, 33, 8), (3, 3, 7, 4), (2, 8, 40, 5)])
+def test_last_token_scores_brute_force(H, Hq, N, d):
+    q = RNG.normal(size=(Hq, d))
+    K = RNG.normal(size=(H, N, d))
+    np.testing.assert_allclose(oracle.last_token_scores(q, K), _brute_last_token(q, K, 1 / math.sqrt(d)),
+                               rtol=1e-12, atol=1e-15)
+
+
+def test_last_token_scores_closed_forms():
+    from scipy.special import softmax
+    # one head: a textbook softmax row; every head's probabilities sum to one => total mass Hq
+    q = RNG.normal(size=(1, 8))
+    K = RNG.normal(size=(1, 25, 8))
+    np.testing.assert_allclose(oracle.last_token_scores(q, K), softmax(K[0] @ q[0] / math.sqrt(8)), rtol=1e-12)
+    q = RNG.normal(size=(6, 8))
+    K = RNG.normal(size=(2, 30, 8))
+    s = oracle.last_token_scores(q, K)
+    assert abs(s.sum() - 6.0) < 1e-12
+    # equal keys: every position gets Hq / N
+    K[:] = K[:, :1, :]
+    np.testing.assert_allclose(oracle.last_token_scores(q, K), np.full(30, 6 / 30), rtol=1e-13)
+    # the grouped-query mapping: head h reads KV head h // G (swap the KV heads <=> swap the query groups)
+    K = RNG.normal(size=(2, 30, 8))
+    a = oracle.last_token_scores(q, K)
+    b = oracle.last_token_scores(np.concatenate([q[3:], q[:3]]), K[::-1])
+    np.testing.assert_allclose(a, b, rtol=1e-13)
+    # agreement with the window scorer's definition for a window of one row
+    win = sum(oracle.window_scores(q[h * 3:(h + 1) * 3, None, :], K[h]) for h in range(2))
+    np.testing.assert_allclose(a[:-1], win, rtol=1e-12)
