@@ -103,8 +103,10 @@ class ClockSampler(threading.Thread):
 
 
 # ------------------------------------------------------------------------------------- roofline per kernel
-def kernel_specs(wl, peaks, sustained: bool):
-    """Algorithmic work of one launch of each kernel of the pass (units of one rank)."""
+def kernel_specs(wl, peaks, sustained: bool, D=None, n_keep=None):
+    """Algorithmic work of one launch of each kernel of the pass (units of one rank).  D and n_keep (width of
+    a hidden-state row, tokens kept) size the kernels of the hidden-state eviction step; without them those
+    entries carry no work figure."""
     u, N, d, P = wl.units, wl.N, wl.d, wl.N - wl.w
     rows, s = wl.G * wl.w, wl.elem_bytes
     tens = peaks["bf16_sustained"] if sustained else peaks["bf16_burst"]
@@ -121,6 +123,11 @@ def kernel_specs(wl, peaks, sustained: bool):
         "eigen_entropy": ("alu", None, None, None),
         "budgets": ("alu", None, None, None),
         "stats_merge": ("hbm", None, None, None),
+        # hidden-state eviction of one layer boundary: keys of one layer in, Hq logits per token out;
+        # logits in, one score per token out; kept rows of the hidden state in and out
+        "evict_logits": ("hbm", (wl.B * wl.H * N * (d * s + wl.G * 4.0)) / 1e9 if D else None, hbm, "GB/s"),
+        "evict_scores": ("hbm", (wl.B * N * (wl.Hq * 4.0 + 4.0)) / 1e9 if D else None, hbm, "GB/s"),
+        "evict_gather": ("hbm", (wl.B * n_keep * (2.0 * D * s + 4.0)) / 1e9 if D else None, hbm, "GB/s"),
     }
 
 
@@ -200,6 +207,155 @@ def _workload_name(wl):
             f"avg budget {wl.avg_budget}, M{wl.M}, n_max {wl.n_max}, k{wl.k_trunc}")
 
 
+# ------------------------------------------------------------------------------- hidden-state eviction
+def run_hidden(args):
+    """One layer-group boundary of the prefill (paper Section 3.3.2): the attention of the last token, summed
+    over the query heads, ranks the positions; the hidden state keeps the best n_keep rows.  Sequences are
+    independent, so ranks are replicas, as for the KV pass."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2410_03090_b200 import binding as ub
+    from paper_2410_03090_b200 import shard, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pass has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group(backend="nccl", device_id=dev)
+    base = synth.scaled(synth.WORKLOADS[args.workload], N=args.scale_N or None, L=1, B=args.hidden_batch)
+    wl = shard.rank_workload(base, rank)
+    D, n_keep = args.hidden_width, wl.N // 2
+    peaks = _peaks()
+    K, _, Qw = synth.generate(wl, dev)
+    Kl = K[:, 0]
+    q = Qw[:, 0, :, -1, :].contiguous()
+    X = synth.hidden_states(wl, D, dev)
+    ctx = ub.Context(ub.make_shape(wl.B, 1, wl.H, wl.Hq, wl.N, wl.d, 1, wl.dtype))
+    scores = torch.empty(wl.B, wl.N - 1, device=dev)
+    idx = torch.empty(wl.B, n_keep, dtype=torch.int32, device=dev)
+    Xout = torch.empty(wl.B, n_keep, D, dtype=X.dtype, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def step(q_, K_, X_):
+        ub.uncomp_evict_hidden(ctx, q_, K_, X_, n_keep, scores=scores, indices=idx, Xout=Xout)
+
+    for _ in range(args.warmup):
+        step(q, Kl, X)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    sampler = ClockSampler(local)
+    sampler.start()
+    ub.uncomp_profile_enable(ctx, True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(q, Kl, X)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    prof = ub.uncomp_profile_read(ctx)
+    ub.uncomp_profile_enable(ctx, False)
+    ms_step = shard.max_over_ranks(ev0.elapsed_time(ev1), dev, world) / args.steps
+    tokens_step = wl.B * wl.N * world
+    specs = kernel_specs(wl, peaks, True, D=D, n_keep=n_keep)
+    kernels, launches = {}, 0
+    total_ms = sum(v[0] for v in prof.values())
+    for name, (ms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        launches += cnt
+        bound, work, peak, unit = specs[name]
+        avg_ms = ms / cnt
+        ent = {"launches_per_step": cnt // args.steps, "avg_ms": round(avg_ms, 5), "share": round(ms / total_ms, 4),
+               "bound": bound}
+        if work is not None:
+            ach = work / (avg_ms / 1e3)
+            ent.update({"achieved": round(ach, 2), "peak": peak, "unit": unit, "frac": round(ach / peak, 4)})
+        kernels[name] = ent
+    dom = max(kernels, key=lambda n: kernels[n]["share"])
+    kd = kernels[dom]
+    roofline = {"kernel": dom, "bound": kd["bound"], "achieved": kd.get("achieved"), "peak": kd.get("peak"),
+                "unit": kd.get("unit"), "frac": kd.get("frac"), "traffic": None,
+                "peak_source": f"of {peaks['source']} (copy)", "avg_ms": kd["avg_ms"], "share": kd["share"]}
+    alg_bytes = sum(specs[n][1] for n in ("evict_logits", "evict_scores", "evict_gather")) * 1e9
+
+    e2e = None
+    if args.e2e_steps > 0:
+        hq = torch.empty(q.shape, dtype=q.dtype, pin_memory=True).copy_(q)
+        hK = torch.empty(Kl.shape, dtype=K.dtype, pin_memory=True).copy_(Kl)
+        hX = torch.empty(X.shape, dtype=X.dtype, pin_memory=True).copy_(X)
+        outs = [idx, Xout]
+        houts = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+        dq, dK, dX = torch.empty_like(hq, device=dev), torch.empty_like(hK, device=dev), torch.empty_like(X)
+
+        def e2e_step():
+            dq.copy_(hq, non_blocking=True)
+            dK.copy_(hK, non_blocking=True)
+            dX.copy_(hX, non_blocking=True)
+            step(dq, dK, dX)
+            for h, t in zip(houts, outs):
+                h.copy_(t, non_blocking=True)
+
+        e2e_step()
+        torch.cuda.synchronize()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+        ms_e = shard.max_over_ranks(e0.elapsed_time(e1), dev, world)
+        e2e = {"value": tokens_step / (ms_e / args.e2e_steps / 1e3), "unit": UNIT,
+               "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in (hq, hK, hX)),
+               "d2h_bytes_per_step": sum(t.numel() * t.element_size() for t in outs), "steps": args.e2e_steps}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        qn, Kn = q[0].double().cpu().numpy(), Kl[0].double().cpu().numpy()
+        rows = X[0].contiguous().view(torch.uint8).reshape(wl.N, -1).cpu().numpy()
+        t0 = time.perf_counter()
+        sc = oracle.last_token_scores(qn, Kn)
+        keep = oracle.select(np.ascontiguousarray(sc[:-1]), 1, n_keep)
+        oracle.compact(rows, keep)
+        t_cpu = time.perf_counter() - t0
+        cpu_baseline = {"value": wl.N / t_cpu, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": f"1 of {wl.B} sequences, whole oracle chain, {t_cpu:.2f} s wall"}
+
+    if rank == 0:
+        line = {"metric": "hidden_state_eviction_tokens_per_s", "value": tokens_step / (ms_step / 1e3), "unit": UNIT,
+                "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
+                "data": "synthetic",
+                "config": {"workload": f"hidden-state eviction at one layer-group boundary: B{wl.B} Hkv{wl.H} "
+                                       f"Hq{wl.Hq} N{wl.N} d{wl.d} D{D} {wl.dtype}, keep {n_keep}",
+                           "l2": f"inputs larger than L2 (keys {Kl.numel() * K.element_size() / 1e9:.2f} GB + hidden "
+                                 f"state {X.numel() * X.element_size() / 1e9:.2f} GB per step)",
+                           "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+                "hbm_pass": {"algorithmic_gb": round(alg_bytes / 1e9, 4),
+                             "achieved_gbs": round(alg_bytes / 1e9 / (ms_step / 1e3), 1),
+                             "frac_of_measured_copy": round(alg_bytes / 1e9 / (ms_step / 1e3) / peaks["hbm_gbs"], 4)},
+                "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
+                "gpu_launches": launches, "clocks": clocks}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ---------------------------------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -212,11 +368,19 @@ def main():
     ap.add_argument("--scale-L", type=int, default=0, help="profiling aid: same recipe with fewer layers")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--path", default="kv", choices=["kv", "hidden"],
+                    help="kv: the KV-cache compression pass (the default and the headline); hidden: the "
+                         "hidden-state eviction of one layer-group boundary, reported on a line of its own")
+    ap.add_argument("--hidden-width", type=int, default=4096)
+    ap.add_argument("--hidden-batch", type=int, default=4)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.path == "hidden":
+        run_hidden(args)
         return
 
     import torch

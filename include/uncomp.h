@@ -239,6 +239,32 @@ int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, unco
 int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_strides sK, uncomp_strides sV,
                    const int32_t *d_indices, const int64_t *d_offsets, void *d_Kc, void *d_Vc, void *stream);
 
+/* ---------------------------------------------------------------------------------------------------
+ * uncomp_evict_hidden -- Section 3.3.2 "Hidden State Eviction" (Algorithm 2: "compress hidden states"):
+ * between layer groups the hidden states of the tokens with the highest attention scores of the LAST token
+ * of the current layer are kept, n_keep of them (the context size d_layer_ctx gives for the next group).
+ *
+ * One layer per call, for every sequence b of the context's shape (L and w of the shape are not used):
+ *   score[j] = sum over the Hq query heads h of softmax_j(scale * <qlast[b,h,:], K[b, h/G, j, :]>), all N positions
+ *   kept = the last position and the n_keep - 1 highest-scored of the first N - 1 (ties: lower position),
+ *          written in ascending order;  Xout[b, t, :] = X[b, kept[t], :]  bit for bit.
+ * Readings where the paper is silent: heads are summed; the last position always survives (it is the
+ * position the next layers continue from).
+ *
+ * d_qlast    in   [B, Hq, d] contiguous, the last position's queries of this layer, storage dtype
+ * d_K        in   this layer's keys [B, H, N, d]; strides sK.sB, sK.sH, sK.sN (sK.sL is ignored)
+ * d_X        in   [B, N, D] contiguous hidden states, storage dtype, D * element size a multiple of 16
+ * n_keep          1 <= n_keep <= N
+ * scale           0 means 1 / sqrt(d)
+ * d_scores   out  [B, N - 1] float scores of the prefix positions; may be NULL
+ * d_indices  out  [B, n_keep] int32
+ * d_Xout     out  [B, n_keep, D]
+ * Rejected: G = Hq / H not in {1, 2, 4, 8, 16} (UNCOMP_E_SHAPE), misaligned rows, n_keep out of range.
+ * ------------------------------------------------------------------------------------------------- */
+int uncomp_evict_hidden(uncomp_ctx *ctx, const void *d_qlast, const void *d_K, uncomp_strides sK, const void *d_X,
+                        int32_t D, int32_t n_keep, float scale, float *d_scores, int32_t *d_indices, void *d_Xout,
+                        void *stream);
+
 /* Synchronise `stream`, copy the status word to *host_bits and clear it on the device.  The only call
  * that waits for the device. */
 int uncomp_status(uncomp_ctx *ctx, void *stream, uint32_t *host_bits);

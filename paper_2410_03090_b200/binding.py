@@ -82,6 +82,8 @@ def _load() -> C.CDLL:
     lib.uncomp_profile_slot_name.argtypes = [C.c_int]
     lib.uncomp_profile_read.restype = C.c_int
     lib.uncomp_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.uncomp_evict_hidden.restype = C.c_int
+    lib.uncomp_evict_hidden.argtypes = [vp, vp, vp, uncomp_strides, vp, C.c_int32, C.c_int32, C.c_float, fp, i32p, vp, vp]
     lib.uncomp_status.restype = C.c_int
     lib.uncomp_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
     return lib
@@ -230,6 +232,23 @@ def uncomp_compact(ctx: Context, K: torch.Tensor, V: torch.Tensor, indices: torc
     _check(lib.uncomp_compact(ctx.handle, _ptr(K), _ptr(V), strides_of(K), strides_of(V), _ptr(indices),
                               _ptr(offsets), _ptr(Kc), _ptr(Vc), _stream(stream)), "uncomp_compact")
     return Kc, Vc
+
+
+def uncomp_evict_hidden(ctx: Context, qlast: torch.Tensor, K_layer: torch.Tensor, X: torch.Tensor, n_keep: int,
+                        scale: float = 0.0, scores: Optional[torch.Tensor] = None,
+                        indices: Optional[torch.Tensor] = None, Xout: Optional[torch.Tensor] = None, stream=None):
+    """qlast [B, Hq, d], K_layer [B, H, N, d] (any 16-byte aligned strides, d contiguous), X [B, N, D]."""
+    B, N, D = X.shape
+    if K_layer.dim() != 4 or K_layer.stride(3) != 1:
+        raise ValueError("expected K_layer [B, H, N, d] with a contiguous last dimension")
+    if indices is None:
+        indices = torch.empty(B, n_keep, dtype=torch.int32, device=X.device)
+    if Xout is None:
+        Xout = torch.empty(B, n_keep, D, dtype=X.dtype, device=X.device)
+    st = uncomp_strides(K_layer.stride(0), 0, K_layer.stride(1), K_layer.stride(2))
+    _check(lib.uncomp_evict_hidden(ctx.handle, _ptr(qlast), _ptr(K_layer), st, _ptr(X), D, n_keep, scale, _ptr(scores),
+                                   _ptr(indices), _ptr(Xout), _stream(stream)), "uncomp_evict_hidden")
+    return indices, Xout
 
 
 def uncomp_status(ctx: Context, stream=None) -> int:

@@ -56,6 +56,12 @@ Plan make_plan(const uncomp_shape &s) {
     p.off_pooled = o;      o = align_up(o + (size_t)p.units * p.prefix * sizeof(float), 256);
     p.off_rank = o;        o = align_up(o + (size_t)p.units * sizeof(int32_t), 256);
     p.off_rem = o;         o = align_up(o + (size_t)p.units * sizeof(int64_t), 256);
+    p.off_ev_logits = o;   o = align_up(o + (size_t)s.B * s.Hq * s.N * sizeof(float), 256);
+    p.off_ev_stats = o;    o = align_up(o + (size_t)s.B * s.Hq * evict_chunks(s) * 2 * sizeof(float), 256);
+    p.off_ev_raw = o;      o = align_up(o + (size_t)s.B * s.N * sizeof(float), 256);
+    p.off_ev_pooled = o;   o = align_up(o + (size_t)s.B * s.N * sizeof(float), 256);
+    p.off_ev_budgets = o;  o = align_up(o + (size_t)s.B * sizeof(int32_t), 256);
+    p.off_ev_offsets = o;  o = align_up(o + (size_t)(s.B + 1) * sizeof(int64_t), 256);
     p.bytes = o;
     return p;
 }
@@ -194,7 +200,8 @@ int uncomp_profile_slots(void) { return kSlotCount; }
 
 const char *uncomp_profile_slot_name(int slot) {
     static const char *names[kSlotCount] = {"gram", "eigen_entropy", "budgets", "score_stats", "stats_merge",
-                                            "score_colsum", "pool_select", "compact", "gram_score_stats"};
+                                            "score_colsum", "pool_select", "compact", "gram_score_stats",
+                                            "evict_logits", "evict_scores", "evict_gather"};
     return slot >= 0 && slot < kSlotCount ? names[slot] : "";
 }
 
@@ -367,6 +374,30 @@ int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_str
         e = launch_compact(p, d_K, d_V, make_addr(p.shape, sK), make_addr(p.shape, sV), d_indices, d_offsets, d_Kc,
                            d_Vc, st);
     }
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+int uncomp_evict_hidden(uncomp_ctx *ctx, const void *d_qlast, const void *d_K, uncomp_strides sK, const void *d_X,
+                        int32_t D, int32_t n_keep, float scale, float *d_scores, int32_t *d_indices, void *d_Xout,
+                        void *stream) {
+    if (!ctx || !d_qlast || !d_K || !d_X || !d_indices || !d_Xout) return UNCOMP_E_NULL;
+    const Plan &p = ctx->plan;
+    const int64_t eb = p.shape.dtype == UNCOMP_FP32 ? 4 : 2;
+    if (!aligned16(d_qlast) || !aligned16(d_K) || !aligned16(d_X) || !aligned16(d_Xout)) return UNCOMP_E_ALIGN;
+    int rc = check_strides(p.shape, sK);
+    if (rc != UNCOMP_OK) return rc;
+    if (D < 1 || ((int64_t)D * eb) % 16 != 0) return UNCOMP_E_ALIGN;
+    if (p.G != 1 && p.G != 2 && p.G != 4 && p.G != 8 && p.G != 16) return UNCOMP_E_SHAPE;
+    if (n_keep < 1 || n_keep > p.shape.N || !(scale >= 0.f) || isinf(scale)) return UNCOMP_E_PARAM;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float *pooled = d_scores ? d_scores : reinterpret_cast<float *>(ctx->ws + p.off_ev_pooled);
+    cudaError_t e = launch_evict_hidden(
+        p, d_qlast, d_K, sK.sB, sK.sH, sK.sN, d_X, (int64_t)D * eb, n_keep, effective_scale(scale, p.shape.d),
+        reinterpret_cast<float *>(ctx->ws + p.off_ev_logits), reinterpret_cast<float *>(ctx->ws + p.off_ev_stats),
+        reinterpret_cast<float *>(ctx->ws + p.off_ev_raw), reinterpret_cast<int32_t *>(ctx->ws + p.off_ev_budgets),
+        reinterpret_cast<int64_t *>(ctx->ws + p.off_ev_offsets), pooled, d_indices, d_Xout,
+        reinterpret_cast<uint32_t *>(ctx->ws + p.off_status), ctx->prof, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;
 }

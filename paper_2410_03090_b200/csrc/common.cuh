@@ -24,6 +24,7 @@ struct Plan {
     int score_splits;   // token chunks per unit in the scorer's statistics pass
     int score_chunk;    // tokens per chunk
     size_t off_status, off_gram, off_stats_part, off_stats, off_raw, off_pooled, off_rank, off_rem;
+    size_t off_ev_logits, off_ev_stats, off_ev_raw, off_ev_pooled, off_ev_budgets, off_ev_offsets;   // hidden-state eviction
     size_t bytes;
 };
 
@@ -62,7 +63,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // Optional per-kernel timing with CUDA events on the launching stream (host objects only).
 enum Slot { kSlotGram = 0, kSlotEigen, kSlotBudgets, kSlotScoreStats, kSlotStatsMerge, kSlotScoreColsum,
-            kSlotPoolSelect, kSlotCompact, kSlotGramStats, kSlotCount };
+            kSlotPoolSelect, kSlotCompact, kSlotGramStats, kSlotEvictLogits, kSlotEvictScores, kSlotEvictGather,
+            kSlotCount };
 enum { kScorePhaseStats = 1, kScorePhaseColsum = 2 };
 struct Profiler;
 void prof_begin(Profiler *p, int slot, cudaStream_t st);
@@ -97,6 +99,11 @@ cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, con
 cudaError_t launch_pool_select(const Plan &p, const float *d_raw, float *d_pooled, int pool_kernel, int pool_mode,
                                const int32_t *d_budgets, const int64_t *d_offsets, int32_t *d_indices,
                                uint32_t *d_status, cudaStream_t st);
+int evict_chunks(const uncomp_shape &s);
+cudaError_t launch_evict_hidden(const Plan &p, const void *d_qlast, const void *d_K, int64_t sB, int64_t sH, int64_t sN,
+                                const void *d_X, int64_t row_bytes, int n_keep, float scale, float *d_logits,
+                                float *d_stats, float *d_raw, int32_t *d_budgets, int64_t *d_offsets, float *d_scores,
+                                int32_t *d_indices, void *d_Xout, uint32_t *d_status, Profiler *prof, cudaStream_t st);
 cudaError_t launch_compact(const Plan &p, const void *dK, const void *dV, const UnitAddr &aK, const UnitAddr &aV,
                            const int32_t *d_indices, const int64_t *d_offsets, void *dKc, void *dVc,
                            cudaStream_t st);

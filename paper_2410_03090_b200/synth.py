@@ -237,6 +237,16 @@ def generate(wl: Workload, device: torch.device | str = "cpu", pin: bool = False
     return K, V, Qw
 
 
+def hidden_states(wl: Workload, D: int, device: torch.device | str = "cpu") -> torch.Tensor:
+    """X [B, N, D]: the residual-stream rows a hidden-state eviction moves (unit-variance noise in the
+    storage dtype; the method only copies these rows, so their values carry no structure)."""
+    g = torch.Generator(device=device).manual_seed(_mix(wl.seed, D, 7) & 0x7FFFFFFF)
+    X = torch.empty(wl.B, wl.N, D, dtype=wl.torch_dtype, device=device)
+    for b in range(wl.B):
+        X[b] = torch.randn(wl.N, D, generator=g, device=device, dtype=torch.float32).to(wl.torch_dtype)
+    return X
+
+
 def unit_index(wl: Workload, u: int) -> Tuple[int, int, int]:
     """(b, l, h) of the flat unit number u (row-major over [B, L, H])."""
     h = u % wl.H
