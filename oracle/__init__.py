@@ -35,6 +35,10 @@ _lib.oracle_window_scores.argtypes = [_dp, _dp, C.c_int, C.c_int, C.c_int, C.c_i
 _lib.oracle_window_scores.restype = None
 _lib.oracle_last_token_scores.argtypes = [_dp, _dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _dp]
 _lib.oracle_last_token_scores.restype = None
+_lib.oracle_decode_probs.argtypes = [_dp, _dp, _dp, C.c_int, C.c_int, C.c_int, C.c_double, _dp]
+_lib.oracle_decode_probs.restype = None
+_lib.oracle_decode_evict.argtypes = [_dp, _i32p, C.c_int, C.c_int, C.c_int]
+_lib.oracle_decode_evict.restype = C.c_int
 _lib.oracle_pool.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _dp]
 _lib.oracle_pool.restype = None
 _lib.oracle_select.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _i32p]
@@ -159,3 +163,46 @@ def last_token_scores(q, K, scale: float | None = None) -> np.ndarray:
     out = np.empty(N, dtype=np.float64)
     _lib.oracle_last_token_scores(_p(q, _dp), _p(K, _dp), H, Hq, N, d, float(scale), _p(out, _dp))
     return out
+
+
+def decode_probs(q, Kc, knew, scale: float | None = None) -> np.ndarray:
+    """Attention of a new token over one head's cache plus itself, summed over the G query heads:
+    q [G, d], Kc [len, d], knew [d] -> p [len + 1]."""
+    q, Kc, knew = _f64(q), _f64(Kc), _f64(knew)
+    G, d = q.shape
+    n = Kc.shape[0]
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    p = np.empty(n + 1, dtype=np.float64)
+    _lib.oracle_decode_probs(_p(q, _dp), _p(Kc, _dp), _p(knew, _dp), G, n, d, float(scale), _p(p, _dp))
+    return p
+
+
+def decode_evict(cum, pos, new_pos: int, protect: int = 1) -> int:
+    """Entry of a full cache that leaves: lowest cumulative score among the entries older than the
+    newest `protect` positions, equal scores to the lower position."""
+    cum = _f64(cum)
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    return int(_lib.oracle_decode_evict(_p(cum, _dp), _p(pos, _i32p), len(cum), int(new_pos), int(protect)))
+
+
+def decode_update(q, Kc, Vc, pos, cum, knew, vnew, new_pos: int, cap: int, protect: int = 1,
+                  scale: float | None = None):
+    """One decode step of one head.  Returns (Kc', Vc', pos', cum', p, evicted position or -1); the cache
+    stays ordered by position (the evicted row is removed, the new token goes to the end)."""
+    Kc, Vc = np.asarray(Kc), np.asarray(Vc)
+    pos = np.asarray(pos, dtype=np.int32)
+    p = decode_probs(q, Kc, knew, scale)
+    n = len(pos)
+    cum2 = _f64(cum) + p[:n]
+    evicted = -1
+    keep = np.ones(n, dtype=bool)
+    if n >= cap:
+        e = decode_evict(cum2, pos, new_pos, protect)
+        evicted = int(pos[e])
+        keep[e] = False
+    K2 = np.concatenate([Kc[keep], np.asarray(knew)[None]], axis=0)
+    V2 = np.concatenate([Vc[keep], np.asarray(vnew)[None]], axis=0)
+    pos2 = np.concatenate([pos[keep], np.array([new_pos], dtype=np.int32)])
+    cum3 = np.concatenate([cum2[keep], p[n:]])
+    return K2, V2, pos2, cum3, p, evicted

@@ -403,3 +403,57 @@ void oracle_last_token_scores(const double *q, const double *K, int H, int Hq, i
     }
     free(s);
 }
+
+/* ----------------------------------------------------------------------------------------------
+ * Decode-time cache update of one head (paper Section 3.3.3, "Dynamic KV Cache Eviction", last sentence;
+ * Algorithm 2, decoding loop): the new token is concatenated with the head's cache, attention is computed
+ * over the concatenation, and once the cache exceeds its budget the entry with the lowest cumulative
+ * attention score is evicted.
+ *
+ * oracle_decode_probs: Kc is the head's cache [len, d], knew [d] the new token's key, q [G, d] the new
+ * token's queries of the G query heads that share this KV head.  Each head's logits scale * (q_g . k_j)
+ * over the len + 1 entries (entry len is the new token) go through a softmax; p[j] is the sum over the G
+ * heads.  p has len + 1 entries.
+ *
+ * oracle_decode_evict: cum [len] are the cumulative scores of the cached entries AFTER this step's p has
+ * been added, pos [len] their positions in the sequence.  Returns the entry to evict: the lowest
+ * cumulative score among the entries with pos <= new_pos - protect (the newest `protect` positions,
+ * the new token included, are not candidates); equal scores: the lower position.  If no entry is a
+ * candidate, every cached entry is one.  len >= 1.
+ * Readings: heads of a group are summed as in the prefill scorer; the new token starts with its own
+ * probability as cumulative score; a cache below its budget appends without evicting (the caller decides).
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_decode_probs(const double *q, const double *Kc, const double *knew, int G, int len, int d,
+                         double scale, double *p)
+{
+    const int n = len + 1;
+    double *s = (double *)malloc((size_t)n * sizeof(double));
+    for (int j = 0; j < n; ++j) p[j] = 0.0;
+    for (int g = 0; g < G; ++g) {
+        const double *qg = q + (size_t)g * d;
+        double mx = -INFINITY;
+        for (int j = 0; j < n; ++j) {
+            const double *k = j < len ? Kc + (size_t)j * d : knew;
+            double acc = 0.0;
+            for (int a = 0; a < d; ++a) acc += qg[a] * k[a];
+            s[j] = scale * acc;
+            if (s[j] > mx) mx = s[j];
+        }
+        double denom = 0.0;
+        for (int j = 0; j < n; ++j) denom += exp(s[j] - mx);
+        for (int j = 0; j < n; ++j) p[j] += exp(s[j] - mx) / denom;
+    }
+    free(s);
+}
+
+int oracle_decode_evict(const double *cum, const int32_t *pos, int len, int new_pos, int protect)
+{
+    int any = 0;
+    for (int j = 0; j < len; ++j) any |= pos[j] <= new_pos - protect;
+    int best = -1;
+    for (int j = 0; j < len; ++j) {
+        if (any && !(pos[j] <= new_pos - protect)) continue;
+        if (best < 0 || cum[j] < cum[best] || (cum[j] == cum[best] && pos[j] < pos[best])) best = j;
+    }
+    return best;
+}
