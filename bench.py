@@ -103,7 +103,7 @@ class ClockSampler(threading.Thread):
 
 
 # ------------------------------------------------------------------------------------- roofline per kernel
-def kernel_specs(wl, peaks, sustained: bool, D=None, n_keep=None):
+def kernel_specs(wl, peaks, sustained: bool, D=None, n_keep=None, cache_rows=None):
     """Algorithmic work of one launch of each kernel of the pass (units of one rank).  D and n_keep (width of
     a hidden-state row, tokens kept) size the kernels of the hidden-state eviction step; without them those
     entries carry no work figure."""
@@ -128,6 +128,11 @@ def kernel_specs(wl, peaks, sustained: bool, D=None, n_keep=None):
         "evict_logits": ("hbm", (wl.B * wl.H * N * (d * s + wl.G * 4.0)) / 1e9 if D else None, hbm, "GB/s"),
         "evict_scores": ("hbm", (wl.B * N * (wl.Hq * 4.0 + 4.0)) / 1e9 if D else None, hbm, "GB/s"),
         "evict_gather": ("hbm", (wl.B * n_keep * (2.0 * D * s + 4.0)) / 1e9 if D else None, hbm, "GB/s"),
+        # decode-time update over cache_rows cached rows: keys in, G logits per row out; logits, cumulative
+        # score and position in, cumulative score out; one new key and value row per unit
+        "decode_logits": ("hbm", cache_rows * (d * s + wl.G * 4.0) / 1e9 if cache_rows else None, hbm, "GB/s"),
+        "decode_accumulate": ("hbm", cache_rows * (wl.G * 4.0 + 12.0) / 1e9 if cache_rows else None, hbm, "GB/s"),
+        "decode_commit": ("hbm", None, None, None),
     }
 
 

@@ -265,6 +265,49 @@ int uncomp_evict_hidden(uncomp_ctx *ctx, const void *d_qlast, const void *d_K, u
                         int32_t D, int32_t n_keep, float scale, float *d_scores, int32_t *d_indices, void *d_Xout,
                         void *stream);
 
+/* ---------------------------------------------------------------------------------------------------
+ * uncomp_decode_update -- Section 3.3.3 "Dynamic KV Cache Eviction", last sentence (as new tokens are
+ * generated, the token with the lowest cumulative attention score is evicted) and Algorithm 2, decoding
+ * loop (the new token is concatenated with each head's cache and attends over the concatenation).
+ *
+ * One decode step for every unit u = (b, l, h) of the context's shape (N and w of the shape are not used
+ * beyond sizing).  Unit u owns rows offsets[u] .. offsets[u+1] - 1 of the ragged cache (the layout
+ * uncomp_compact writes: its capacity is the head's token budget) of which the first lens[u] are filled.
+ *   p[j]   = sum over the G query heads g of softmax_j(scale * <qnew[u*G+g, :], k_j>), j over the lens[u]
+ *            cached keys and, as entry lens[u], the new token's own key
+ *   cum[j] += p[j] for the cached entries; the new token's cumulative score starts at p[lens[u]]
+ *   lens[u] <  capacity: the new token is appended, lens[u] += 1, evicted[u] = -1
+ *   lens[u] == capacity: the cached entry with the lowest cum among those with pos <= new_pos[b] - protect
+ *            leaves (equal scores: the lower position; no such entry: all cached entries are candidates),
+ *            evicted[u] = its position, and the new token takes its ROW: rows of a unit are not kept in
+ *            position order, d_pos names the position of each row.
+ * Readings where the paper is silent: grouped query heads are summed as in the prefill scorer; the new
+ * token cannot leave in the step that adds it (protect >= 1 newest positions are never candidates).
+ *
+ * d_qnew     in      [B, L, Hq, d] contiguous, storage dtype: the new token's queries
+ * d_knew     in      [B, L, H, d] contiguous; d_vnew likewise: the new token's key and value rows
+ * d_new_pos  in      [B] int32, the new token's position in its sequence (larger than every cached pos)
+ * d_offsets  in      [B*L*H + 1] int64
+ * d_lens     in/out  [B*L*H] int32
+ * max_cap            host: an upper bound of every unit's capacity, 1 <= max_cap <= N (sizes the grid)
+ * total_cap          host: offsets[B*L*H]
+ * protect            >= 1
+ * scale              0 means 1 / sqrt(d)
+ * d_Kc, d_Vc in/out  [total_cap, d] storage dtype, 16-byte aligned
+ * d_pos      in/out  [total_cap] int32
+ * d_cum      in/out  [total_cap] float
+ * d_p        out     [total_cap + B*L*H] float, entry j of unit u at offsets[u] + u + j; may be NULL
+ * d_evicted  out     [B*L*H] int32; may be NULL
+ * Rejected: G not in {1, 2, 4, 8, 16} (UNCOMP_E_SHAPE); (total_cap + units) * G floats beyond the
+ * workspace region that holds the logits, 2 * units * (N - w) floats (UNCOMP_E_LIMIT).  A unit whose
+ * capacity is 0 or above max_cap, or whose length is outside [0, capacity], is left untouched and raises
+ * UNCOMP_STATUS_BOUNDS.
+ * ------------------------------------------------------------------------------------------------- */
+int uncomp_decode_update(uncomp_ctx *ctx, const void *d_qnew, const void *d_knew, const void *d_vnew,
+                         const int32_t *d_new_pos, const int64_t *d_offsets, int32_t *d_lens, int32_t max_cap,
+                         int64_t total_cap, int32_t protect, float scale, void *d_Kc, void *d_Vc, int32_t *d_pos,
+                         float *d_cum, float *d_p, int32_t *d_evicted, void *stream);
+
 /* Synchronise `stream`, copy the status word to *host_bits and clear it on the device.  The only call
  * that waits for the device. */
 int uncomp_status(uncomp_ctx *ctx, void *stream, uint32_t *host_bits);

@@ -82,6 +82,9 @@ def _load() -> C.CDLL:
     lib.uncomp_profile_slot_name.argtypes = [C.c_int]
     lib.uncomp_profile_read.restype = C.c_int
     lib.uncomp_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.uncomp_decode_update.restype = C.c_int
+    lib.uncomp_decode_update.argtypes = [vp, vp, vp, vp, i32p, i64p, i32p, C.c_int32, C.c_int64, C.c_int32, C.c_float,
+                                         vp, vp, i32p, fp, fp, i32p, vp]
     lib.uncomp_evict_hidden.restype = C.c_int
     lib.uncomp_evict_hidden.argtypes = [vp, vp, vp, uncomp_strides, vp, C.c_int32, C.c_int32, C.c_float, fp, i32p, vp, vp]
     lib.uncomp_status.restype = C.c_int
@@ -249,6 +252,19 @@ def uncomp_evict_hidden(ctx: Context, qlast: torch.Tensor, K_layer: torch.Tensor
     _check(lib.uncomp_evict_hidden(ctx.handle, _ptr(qlast), _ptr(K_layer), st, _ptr(X), D, n_keep, scale, _ptr(scores),
                                    _ptr(indices), _ptr(Xout), _stream(stream)), "uncomp_evict_hidden")
     return indices, Xout
+
+
+def uncomp_decode_update(ctx: Context, qnew: torch.Tensor, knew: torch.Tensor, vnew: torch.Tensor,
+                         new_pos: torch.Tensor, offsets: torch.Tensor, lens: torch.Tensor, max_cap: int,
+                         Kc: torch.Tensor, Vc: torch.Tensor, pos: torch.Tensor, cum: torch.Tensor, protect: int = 1,
+                         scale: float = 0.0, p: Optional[torch.Tensor] = None,
+                         evicted: Optional[torch.Tensor] = None, stream=None):
+    """One decode step on the ragged cache, in place: qnew [B, L, Hq, d], knew / vnew [B, L, H, d],
+    new_pos [B] int32, offsets [units + 1] int64, lens [units] int32, Kc / Vc [total_cap, d], pos int32 and
+    cum float32 [total_cap]; optional outputs p [total_cap + units] and evicted [units]."""
+    _check(lib.uncomp_decode_update(ctx.handle, _ptr(qnew), _ptr(knew), _ptr(vnew), _ptr(new_pos), _ptr(offsets),
+                                    _ptr(lens), max_cap, Kc.shape[0], protect, scale, _ptr(Kc), _ptr(Vc), _ptr(pos),
+                                    _ptr(cum), _ptr(p), _ptr(evicted), _stream(stream)), "uncomp_decode_update")
 
 
 def uncomp_status(ctx: Context, stream=None) -> int:

@@ -62,6 +62,9 @@ Plan make_plan(const uncomp_shape &s) {
     p.off_ev_pooled = o;   o = align_up(o + (size_t)s.B * s.N * sizeof(float), 256);
     p.off_ev_budgets = o;  o = align_up(o + (size_t)s.B * sizeof(int32_t), 256);
     p.off_ev_offsets = o;  o = align_up(o + (size_t)(s.B + 1) * sizeof(int64_t), 256);
+    p.off_dec_stats = o;   o = align_up(o + (size_t)p.units * decode_chunks(s.N) * 16 * 2 * sizeof(float), 256);
+    p.off_dec_part = o;    o = align_up(o + (size_t)p.units * decode_chunks(s.N) * decode_partial_bytes(), 256);
+    p.off_dec_new = o;     o = align_up(o + (size_t)p.units * sizeof(float), 256);
     p.bytes = o;
     return p;
 }
@@ -201,7 +204,8 @@ int uncomp_profile_slots(void) { return kSlotCount; }
 const char *uncomp_profile_slot_name(int slot) {
     static const char *names[kSlotCount] = {"gram", "eigen_entropy", "budgets", "score_stats", "stats_merge",
                                             "score_colsum", "pool_select", "compact", "gram_score_stats",
-                                            "evict_logits", "evict_scores", "evict_gather"};
+                                            "evict_logits", "evict_scores", "evict_gather",
+                                            "decode_logits", "decode_accumulate", "decode_commit"};
     return slot >= 0 && slot < kSlotCount ? names[slot] : "";
 }
 
@@ -374,6 +378,32 @@ int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_str
         e = launch_compact(p, d_K, d_V, make_addr(p.shape, sK), make_addr(p.shape, sV), d_indices, d_offsets, d_Kc,
                            d_Vc, st);
     }
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+int uncomp_decode_update(uncomp_ctx *ctx, const void *d_qnew, const void *d_knew, const void *d_vnew,
+                         const int32_t *d_new_pos, const int64_t *d_offsets, int32_t *d_lens, int32_t max_cap,
+                         int64_t total_cap, int32_t protect, float scale, void *d_Kc, void *d_Vc, int32_t *d_pos,
+                         float *d_cum, float *d_p, int32_t *d_evicted, void *stream) {
+    if (!ctx || !d_qnew || !d_knew || !d_vnew || !d_new_pos || !d_offsets || !d_lens || !d_Kc || !d_Vc || !d_pos ||
+        !d_cum)
+        return UNCOMP_E_NULL;
+    const Plan &p = ctx->plan;
+    if (!aligned16(d_qnew) || !aligned16(d_knew) || !aligned16(d_vnew) || !aligned16(d_Kc) || !aligned16(d_Vc))
+        return UNCOMP_E_ALIGN;
+    if (p.G != 1 && p.G != 2 && p.G != 4 && p.G != 8 && p.G != 16) return UNCOMP_E_SHAPE;
+    if (max_cap < 1 || max_cap > p.shape.N || total_cap < 1 || protect < 1 || !(scale >= 0.f) || isinf(scale))
+        return UNCOMP_E_PARAM;
+    // the logits of every entry live in the region the prefill pass uses for its raw and pooled scores
+    if ((size_t)(total_cap + p.units) * p.G * sizeof(float) > p.off_rank - p.off_raw) return UNCOMP_E_LIMIT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_decode_update(
+        p, d_qnew, d_knew, d_vnew, d_new_pos, d_offsets, d_lens, max_cap, protect, effective_scale(scale, p.shape.d),
+        d_Kc, d_Vc, d_pos, d_cum, d_p, d_evicted, reinterpret_cast<float *>(ctx->ws + p.off_raw),
+        reinterpret_cast<float *>(ctx->ws + p.off_dec_stats), ctx->ws + p.off_dec_part,
+        reinterpret_cast<float *>(ctx->ws + p.off_dec_new), reinterpret_cast<uint32_t *>(ctx->ws + p.off_status),
+        ctx->prof, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;
 }

@@ -25,6 +25,7 @@ struct Plan {
     int score_chunk;    // tokens per chunk
     size_t off_status, off_gram, off_stats_part, off_stats, off_raw, off_pooled, off_rank, off_rem;
     size_t off_ev_logits, off_ev_stats, off_ev_raw, off_ev_pooled, off_ev_budgets, off_ev_offsets;   // hidden-state eviction
+    size_t off_dec_stats, off_dec_part, off_dec_new;   // decode-time update (its logits reuse off_raw .. off_rank)
     size_t bytes;
 };
 
@@ -64,7 +65,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // Optional per-kernel timing with CUDA events on the launching stream (host objects only).
 enum Slot { kSlotGram = 0, kSlotEigen, kSlotBudgets, kSlotScoreStats, kSlotStatsMerge, kSlotScoreColsum,
             kSlotPoolSelect, kSlotCompact, kSlotGramStats, kSlotEvictLogits, kSlotEvictScores, kSlotEvictGather,
-            kSlotCount };
+            kSlotDecodeLogits, kSlotDecodeAccumulate, kSlotDecodeCommit, kSlotCount };
 enum { kScorePhaseStats = 1, kScorePhaseColsum = 2 };
 struct Profiler;
 void prof_begin(Profiler *p, int slot, cudaStream_t st);
@@ -104,6 +105,13 @@ cudaError_t launch_evict_hidden(const Plan &p, const void *d_qlast, const void *
                                 const void *d_X, int64_t row_bytes, int n_keep, float scale, float *d_logits,
                                 float *d_stats, float *d_raw, int32_t *d_budgets, int64_t *d_offsets, float *d_scores,
                                 int32_t *d_indices, void *d_Xout, uint32_t *d_status, Profiler *prof, cudaStream_t st);
+int decode_chunks(int max_cap);
+size_t decode_partial_bytes();
+cudaError_t launch_decode_update(const Plan &p, const void *d_q, const void *d_knew, const void *d_vnew,
+                                 const int32_t *d_new_pos, const int64_t *d_offsets, int32_t *d_lens, int max_cap,
+                                 int protect, float scale, void *d_Kc, void *d_Vc, int32_t *d_pos, float *d_cum,
+                                 float *d_p, int32_t *d_evicted, float *d_logits, float *d_stats, void *d_partial,
+                                 float *d_new_cum, uint32_t *d_status, Profiler *prof, cudaStream_t st);
 cudaError_t launch_compact(const Plan &p, const void *dK, const void *dV, const UnitAddr &aK, const UnitAddr &aV,
                            const int32_t *d_indices, const int64_t *d_offsets, void *dKc, void *dVc,
                            cudaStream_t st);
