@@ -361,6 +361,177 @@ def run_hidden(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------ decode-time update
+def run_decode(args):
+    """One decode step over the compressed cache of every layer (paper Section 3.3.3, last sentence of "Dynamic
+    KV Cache Eviction"): the prefill pass builds the ragged cache, then every timed step appends one token per
+    sequence to every head's cache and evicts the entry with the lowest cumulative score."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2410_03090_b200 import binding as ub
+    from paper_2410_03090_b200 import shard, synth
+    from paper_2410_03090_b200.compress import CompressionPass
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pass has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group(backend="nccl", device_id=dev)
+    base = synth.WORKLOADS[args.workload]
+    if args.scale_N or args.scale_L:
+        base = synth.scaled(base, N=args.scale_N or None, L=args.scale_L or None)
+    wl = shard.rank_workload(base, rank)
+    peaks = _peaks()
+    K, V, Qw = synth.generate(wl, dev)
+    cp = CompressionPass(wl, dev)
+    o = cp.run(K, V, Qw)
+    torch.cuda.synchronize()
+    assert cp.status() == 0
+    # state after prefill: full caches; cumulative scores seeded with the prefill scores of the kept prefix
+    # tokens and, for the window tokens (which the prefill does not score), the largest of them
+    offs = o.offsets.cpu().numpy()
+    P = wl.N - wl.w
+    cum = torch.empty(wl.total_rows, device=dev)
+    sc = o.scores.view(wl.units, P)
+    for u in range(wl.units):
+        idx = o.indices[offs[u]:offs[u + 1]].long()
+        pre = idx < P
+        cum[offs[u]:offs[u + 1]] = torch.where(pre, sc[u][idx.clamp(max=P - 1)], sc[u].max())
+    pos = o.indices.clone()
+    lens = o.budgets.reshape(-1).clone()
+    Kc, Vc = o.Kc, o.Vc
+    max_cap = int(lens.max())
+    qnew = Qw[:, :, :, -1, :].contiguous()
+    knew = K[:, :, :, -1, :].contiguous()
+    vnew = V[:, :, :, -1, :].contiguous()
+    del K, V
+    n_steps = args.warmup + args.steps + args.e2e_steps + 2
+    new_pos = [torch.full((wl.B,), wl.N + i, dtype=torch.int32, device=dev) for i in range(n_steps)]
+    evicted = torch.empty(wl.units, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    it = iter(new_pos)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def step(q_, k_, v_):
+        ub.uncomp_decode_update(cp.ctx, q_, k_, v_, next(it), o.offsets, lens, max_cap, Kc, Vc, pos, cum,
+                                evicted=evicted)
+
+    for _ in range(args.warmup):
+        step(qnew, knew, vnew)
+    torch.cuda.synchronize()
+    assert cp.status() == 0
+    sampler = ClockSampler(local)
+    sampler.start()
+    ub.uncomp_profile_enable(cp.ctx, True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(qnew, knew, vnew)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    prof = ub.uncomp_profile_read(cp.ctx)
+    ub.uncomp_profile_enable(cp.ctx, False)
+    ms_step = shard.max_over_ranks(ev0.elapsed_time(ev1), dev, world) / args.steps
+    tokens_step = wl.B * world
+    specs = kernel_specs(wl, peaks, True, cache_rows=wl.total_rows)
+    kernels, launches = {}, 0
+    total_ms = sum(v[0] for v in prof.values())
+    for name, (ms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        launches += cnt
+        bound, work, peak, unit = specs[name]
+        avg_ms = ms / cnt
+        ent = {"launches_per_step": cnt // args.steps, "avg_ms": round(avg_ms, 5), "share": round(ms / total_ms, 4),
+               "bound": bound}
+        if work is not None:
+            ach = work / (avg_ms / 1e3)
+            ent.update({"achieved": round(ach, 2), "peak": peak, "unit": unit, "frac": round(ach / peak, 4)})
+        kernels[name] = ent
+    dom = max(kernels, key=lambda n: kernels[n]["share"])
+    kd = kernels[dom]
+    roofline = {"kernel": dom, "bound": kd["bound"], "achieved": kd.get("achieved"), "peak": kd.get("peak"),
+                "unit": kd.get("unit"), "frac": kd.get("frac"), "traffic": None,
+                "peak_source": f"of {peaks['source']} (copy)", "avg_ms": kd["avg_ms"], "share": kd["share"]}
+    alg_bytes = (specs["decode_logits"][1] + specs["decode_accumulate"][1]) * 1e9
+
+    e2e = None
+    if args.e2e_steps > 0:
+        hin = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for t in (qnew, knew, vnew)]
+        din = [torch.empty_like(t) for t in (qnew, knew, vnew)]
+        hev = torch.empty(evicted.shape, dtype=evicted.dtype, pin_memory=True)
+
+        def e2e_step():
+            for h, t in zip(hin, din):
+                t.copy_(h, non_blocking=True)
+            step(*din)
+            hev.copy_(evicted, non_blocking=True)
+
+        e2e_step()
+        torch.cuda.synchronize()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+        ms_e = shard.max_over_ranks(e0.elapsed_time(e1), dev, world)
+        e2e = {"value": tokens_step / (ms_e / args.e2e_steps / 1e3), "unit": UNIT,
+               "h2d_bytes_per_step": sum(t.numel() * t.element_size() for t in hin),
+               "d2h_bytes_per_step": hev.numel() * hev.element_size(), "steps": args.e2e_steps}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        sample = list(range(0, wl.units, max(1, wl.units // 16)))[:16]
+        data = []
+        for u in sample:
+            a, b = int(offs[u]), int(offs[u + 1])
+            data.append((qnew.view(wl.units, wl.G, wl.d)[u].double().cpu().numpy(), Kc[a:b].double().cpu().numpy(),
+                         Vc[a:b].double().cpu().numpy(), pos[a:b].cpu().numpy(), cum[a:b].double().cpu().numpy(),
+                         knew.view(wl.units, wl.d)[u].double().cpu().numpy(),
+                         vnew.view(wl.units, wl.d)[u].double().cpu().numpy(), b - a))
+        t0 = time.perf_counter()
+        for q_, K_, V_, p_, c_, kn_, vn_, cap in data:
+            oracle.decode_update(q_, K_, V_, p_, c_, kn_, vn_, wl.N + n_steps, cap)
+        t_cpu = time.perf_counter() - t0
+        cpu_baseline = {"value": wl.B / (t_cpu * wl.units / len(sample)), "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": f"{len(sample)} of {wl.units} units, one decode step, {t_cpu:.2f} s wall"}
+
+    if rank == 0:
+        line = {"metric": "decode_cache_update_tokens_per_s", "value": tokens_step / (ms_step / 1e3), "unit": UNIT,
+                "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
+                "data": "synthetic",
+                "config": {"workload": f"decode-time cache update after the prefill pass of {_workload_name(wl)}: "
+                                       f"{wl.units} head caches, {wl.total_rows} cached rows, largest {max_cap}",
+                           "l2": f"cached keys {wl.total_rows * wl.d * wl.elem_bytes / 1e9:.3f} GB read every step"
+                                 + ("" if wl.total_rows * wl.d * wl.elem_bytes > 126e6 else " (fits in L2)"),
+                           "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+                "hbm_pass": {"algorithmic_gb": round(alg_bytes / 1e9, 4),
+                             "achieved_gbs": round(alg_bytes / 1e9 / (ms_step / 1e3), 1),
+                             "frac_of_measured_copy": round(alg_bytes / 1e9 / (ms_step / 1e3) / peaks["hbm_gbs"], 4)},
+                "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
+                "gpu_launches": launches, "clocks": clocks}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ---------------------------------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -373,9 +544,10 @@ def main():
     ap.add_argument("--scale-L", type=int, default=0, help="profiling aid: same recipe with fewer layers")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--path", default="kv", choices=["kv", "hidden"],
+    ap.add_argument("--path", default="kv", choices=["kv", "hidden", "decode"],
                     help="kv: the KV-cache compression pass (the default and the headline); hidden: the "
-                         "hidden-state eviction of one layer-group boundary, reported on a line of its own")
+                         "hidden-state eviction of one layer-group boundary; decode: one decode-time update of "
+                         "the compressed cache of every layer; each reported on a line of its own")
     ap.add_argument("--hidden-width", type=int, default=4096)
     ap.add_argument("--hidden-batch", type=int, default=4)
     args = ap.parse_args()
@@ -386,6 +558,9 @@ def main():
         return
     if args.path == "hidden":
         run_hidden(args)
+        return
+    if args.path == "decode":
+        run_decode(args)
         return
 
     import torch

@@ -251,8 +251,19 @@ __global__ void __launch_bounds__(kDecThreads) decode_accumulate_kernel(DecArgs 
     best.el.j = best.any.j = -1;
     const int t1 = min(n, (c + 1) * kDecChunk);
     for (int j = c * kDecChunk + tid; j < t1; j += kDecThreads) {
-        float p = 0.f;
-        for (int g = 0; g < G; ++g) p += ex2f(lg[(int64_t)j * G + g] - mprime[g]);
+        float p = 0.f;   // heads in ascending order, whichever load width is used
+        if ((G & 3) == 0) {
+            const float4 *l4 = reinterpret_cast<const float4 *>(lg + (int64_t)j * G);
+            for (int g = 0; g < G; g += 4) {
+                const float4 x = l4[g >> 2];
+                p += ex2f(x.x - mprime[g]);
+                p += ex2f(x.y - mprime[g + 1]);
+                p += ex2f(x.z - mprime[g + 2]);
+                p += ex2f(x.w - mprime[g + 3]);
+            }
+        } else {
+            for (int g = 0; g < G; ++g) p += ex2f(lg[(int64_t)j * G + g] - mprime[g]);
+        }
         if (p_out) p_out[off + u + j] = p;
         if (j < len) {
             const float cn = cum[off + j] + p;
