@@ -39,6 +39,12 @@ _lib.oracle_decode_probs.argtypes = [_dp, _dp, _dp, C.c_int, C.c_int, C.c_int, C
 _lib.oracle_decode_probs.restype = None
 _lib.oracle_decode_evict.argtypes = [_dp, _i32p, C.c_int, C.c_int, C.c_int]
 _lib.oracle_decode_evict.restype = C.c_int
+_lib.oracle_prepare_mean.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _dp]
+_lib.oracle_prepare_mean.restype = None
+_lib.oracle_group_labels.argtypes = [_dp, C.c_int, C.c_int, C.c_int, C.c_int, _i32p]
+_lib.oracle_group_labels.restype = C.c_int
+_lib.oracle_majority_vote.argtypes = [_dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, _i32p, _i32p]
+_lib.oracle_majority_vote.restype = C.c_int
 _lib.oracle_pool.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _dp]
 _lib.oracle_pool.restype = None
 _lib.oracle_select.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _i32p]
@@ -206,3 +212,33 @@ def decode_update(q, Kc, Vc, pos, cum, knew, vnew, new_pos: int, cap: int, prote
     pos2 = np.concatenate([pos[keep], np.array([new_pos], dtype=np.int32)])
     cum3 = np.concatenate([cum2[keep], p[n:]])
     return K2, V2, pos2, cum3, p, evicted
+
+
+def prepare_mean(erank) -> np.ndarray:
+    """Averaged effective rank over the samples: erank [S, L, H] -> [L, H]."""
+    erank = _f64(erank)
+    S, L, H = erank.shape
+    out = np.empty((L, H), dtype=np.float64)
+    _lib.oracle_prepare_mean(_p(erank, _dp), S, L, H, _p(out, _dp))
+    return out
+
+
+def group_labels(values, M: int, scope: int = 0) -> np.ndarray:
+    """Rank-based group of every head: values [L, H] -> int32 [L, H], group 0 the highest values."""
+    values = _f64(values)
+    L, H = values.shape
+    out = np.empty((L, H), dtype=np.int32)
+    if _lib.oracle_group_labels(_p(values, _dp), L, H, int(M), int(scope), _p(out, _i32p)) != 0:
+        raise ValueError("M must be between 1 and the size of the ranking set")
+    return out
+
+
+def majority_vote(erank, M: int, scope: int = 0):
+    """Per-sample grouping and majority vote: erank [S, L, H] -> (votes int32 [L, H, M], labels int32 [L, H])."""
+    erank = _f64(erank)
+    S, L, H = erank.shape
+    votes = np.empty((L, H, M), dtype=np.int32)
+    labels = np.empty((L, H), dtype=np.int32)
+    if _lib.oracle_majority_vote(_p(erank, _dp), S, L, H, int(M), int(scope), _p(votes, _i32p), _p(labels, _i32p)) != 0:
+        raise ValueError("M must be between 1 and the size of the ranking set")
+    return votes, labels

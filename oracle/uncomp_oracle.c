@@ -457,3 +457,69 @@ int oracle_decode_evict(const double *cum, const int32_t *pos, int len, int new_
     }
     return best;
 }
+
+/* ----------------------------------------------------------------------------------------------
+ * Preparation stage (Section 3.3.1 "Preparation Stage", its equation for the averaged effective rank;
+ * Algorithm 1, head group identification).
+ *
+ * erank is [S, L, H]: the truncated effective rank of every head for each of S samples.
+ *   oracle_prepare_mean    mean[l,h] = (1/S) sum_i erank[i,l,h]                       (the equation)
+ *   oracle_group_labels    heads of a ranking set (one layer: scope 0, n = H; the whole model: scope 1,
+ *                          n = L*H) sorted by descending value, equal values by ascending index; the head
+ *                          at rank r gets group g with floor(g n / M) <= r < floor((g+1) n / M): M groups
+ *                          whose sizes differ by at most one, group 0 the highest values (the grouping
+ *                          the budget rule uses).  values is [L, H], one label per head.
+ *   oracle_majority_vote   Algorithm 1: every sample labels the heads by oracle_group_labels on its own
+ *                          values; votes[l,h,g] counts the samples that put head (l,h) in group g; the
+ *                          final label is the group with most votes, the lowest such group on a tie.
+ * Readings: "one of 8 clusters based on E" is taken as the rank-based equal-size grouping above (the
+ * paper names no clustering algorithm and the inference stage ranks heads the same way); M = 2 gives
+ * the retrieval / streaming split of Section 3.3.3 "Retrieval Head" with label 0 the retrieval heads.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_prepare_mean(const double *erank, int S, int L, int H, double *mean)
+{
+    for (int i = 0; i < L * H; ++i) {
+        double acc = 0.0;
+        for (int s = 0; s < S; ++s) acc += erank[(size_t)s * L * H + i];
+        mean[i] = acc / (double)S;
+    }
+}
+
+int oracle_group_labels(const double *values, int L, int H, int M, int scope, int32_t *labels)
+{
+    const int n = scope ? L * H : H;
+    const int sets = scope ? 1 : L;
+    if (M < 1 || M > n) return -1;
+    keyed_t *order = (keyed_t *)malloc((size_t)n * sizeof(keyed_t));
+    for (int s = 0; s < sets; ++s) {
+        const size_t base = (size_t)s * n;
+        for (int i = 0; i < n; ++i) { order[i].key = values[base + i]; order[i].idx = i; }
+        qsort(order, (size_t)n, sizeof(keyed_t), cmp_key_desc_idx_asc);
+        for (int g = 0; g < M; ++g) {
+            const int lo = (int)((int64_t)g * n / M), hi = (int)((int64_t)(g + 1) * n / M);
+            for (int r = lo; r < hi; ++r) labels[base + order[r].idx] = g;
+        }
+    }
+    free(order);
+    return 0;
+}
+
+int oracle_majority_vote(const double *erank, int S, int L, int H, int M, int scope, int32_t *votes,
+                         int32_t *labels)
+{
+    const int LH = L * H;
+    int32_t *one = (int32_t *)malloc((size_t)LH * sizeof(int32_t));
+    for (int i = 0; i < LH * M; ++i) votes[i] = 0;
+    for (int s = 0; s < S; ++s) {
+        if (oracle_group_labels(erank + (size_t)s * LH, L, H, M, scope, one) != 0) { free(one); return -1; }
+        for (int i = 0; i < LH; ++i) votes[(size_t)i * M + one[i]] += 1;
+    }
+    for (int i = 0; i < LH; ++i) {
+        int best = 0;
+        for (int g = 1; g < M; ++g)
+            if (votes[(size_t)i * M + g] > votes[(size_t)i * M + best]) best = g;
+        labels[i] = best;
+    }
+    free(one);
+    return 0;
+}
