@@ -133,6 +133,8 @@ def kernel_specs(wl, peaks, sustained: bool, D=None, n_keep=None, cache_rows=Non
         "decode_logits": ("hbm", cache_rows * (d * s + wl.G * 4.0) / 1e9 if cache_rows else None, hbm, "GB/s"),
         "decode_accumulate": ("hbm", cache_rows * (wl.G * 4.0 + 12.0) / 1e9 if cache_rows else None, hbm, "GB/s"),
         "decode_commit": ("hbm", None, None, None),
+        "prepare_vote": ("alu", None, None, None),
+        "prepare_finish": ("alu", None, None, None),
     }
 
 
@@ -532,6 +534,85 @@ def run_decode(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------ preparation stage
+def run_prepare(args):
+    """Aggregation of the preparation stage (paper Section 3.3.1; Algorithm 1) over 500 samples' effective ranks
+    for the workload's layers and heads: mean, grouping of the mean, per-sample grouping and majority vote.
+    Latency-bound integer work on 0.5 MB; single GPU only."""
+    import numpy as np
+    import torch
+    from paper_2410_03090_b200 import binding as ub
+    from paper_2410_03090_b200 import synth
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pass has no CPU path")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    wl = synth.WORKLOADS[args.workload]
+    S, M = 500, min(8, wl.H)
+    g = torch.Generator(device=dev).manual_seed(wl.seed)
+    erank = (torch.rand(wl.L, wl.H, generator=g, device=dev) * 30 + 1)[None] + \
+        torch.randn(S, wl.L, wl.H, generator=g, device=dev) * 2.0
+    ctx = ub.Context(ub.make_shape(1, wl.L, wl.H, wl.Hq, 256, wl.d, 8, wl.dtype))
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        ub.uncomp_prepare_groups(ctx, erank, M, 0)
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    ub.uncomp_profile_enable(ctx, True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        out = ub.uncomp_prepare_groups(ctx, erank, M, 0)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    prof = ub.uncomp_profile_read(ctx)
+    ms_step = ev0.elapsed_time(ev1) / args.steps
+    kernels = {n: {"launches_per_step": c // args.steps, "avg_ms": round(ms / c, 5), "bound": "alu"}
+               for n, (ms, c) in prof.items() if c}
+    launches = sum(c for _, c in prof.values())
+    h = torch.empty(erank.shape, dtype=erank.dtype, pin_memory=True).copy_(erank)
+    d_in = torch.empty_like(erank)
+    houts = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in out]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(max(1, args.e2e_steps)):
+        d_in.copy_(h, non_blocking=True)
+        res = ub.uncomp_prepare_groups(ctx, d_in, M, 0)
+        for a, b in zip(houts, res):
+            a.copy_(b, non_blocking=True)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_e = e0.elapsed_time(e1) / max(1, args.e2e_steps)
+    import oracle
+    e64 = erank.double().cpu().numpy()
+    t0 = time.perf_counter()
+    oracle.group_labels(oracle.prepare_mean(e64), M)
+    oracle.majority_vote(e64, M)
+    t_cpu = time.perf_counter() - t0
+    dom = max(kernels, key=lambda n: kernels[n]["avg_ms"])
+    line = {"metric": "preparation_aggregation_samples_per_s", "value": S / (ms_step / 1e3), "unit": "samples/s",
+            "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"preparation-stage aggregation: S{S} samples x L{wl.L} x H{wl.H} effective ranks, "
+                                   f"M{M} groups per layer", "l2": "0.5 MB of input: resident in L2, latency-bound"},
+            "roofline": {"kernel": dom, "bound": "alu", "achieved": None, "peak": None, "unit": None, "frac": None,
+                         "traffic": None, "avg_ms": kernels[dom]["avg_ms"],
+                         "note": "two launches of a few microseconds each; no throughput roofline applies"},
+            "kernels": kernels,
+            "cpu_baseline": {"value": S / t_cpu, "unit": "samples/s", "cores": 1, "kind": "oracle",
+                             "sample": f"the whole aggregation, {t_cpu * 1e3:.1f} ms wall"},
+            "e2e": {"value": S / (ms_e / 1e3), "unit": "samples/s", "h2d_bytes_per_step": h.numel() * 4,
+                    "d2h_bytes_per_step": sum(t.numel() * t.element_size() for t in out)},
+            "gpu_launches": launches, "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
 # ---------------------------------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -544,7 +625,7 @@ def main():
     ap.add_argument("--scale-L", type=int, default=0, help="profiling aid: same recipe with fewer layers")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--path", default="kv", choices=["kv", "hidden", "decode"],
+    ap.add_argument("--path", default="kv", choices=["kv", "hidden", "decode", "prepare"],
                     help="kv: the KV-cache compression pass (the default and the headline); hidden: the "
                          "hidden-state eviction of one layer-group boundary; decode: one decode-time update of "
                          "the compressed cache of every layer; each reported on a line of its own")
@@ -561,6 +642,9 @@ def main():
         return
     if args.path == "decode":
         run_decode(args)
+        return
+    if args.path == "prepare":
+        run_prepare(args)
         return
 
     import torch

@@ -308,6 +308,32 @@ int uncomp_decode_update(uncomp_ctx *ctx, const void *d_qnew, const void *d_knew
                          int64_t total_cap, int32_t protect, float scale, void *d_Kc, void *d_Vc, int32_t *d_pos,
                          float *d_cum, float *d_p, int32_t *d_evicted, void *stream);
 
+/* ---------------------------------------------------------------------------------------------------
+ * uncomp_prepare_groups -- Section 3.3.1 "Preparation Stage" (the effective rank of each head averaged
+ * over the d sampled data points) and Algorithm 1 (each sample assigns every head to one of M clusters by
+ * its truncated entropy; the final label of a head is the majority vote).  With M = 2 the labels are the
+ * retrieval / streaming split of Section 3.3.3 "Retrieval Head" (label 0: the high-rank group).
+ *
+ * L and H come from the context's shape.  A ranking set is one layer (scope 0, n = H) or the whole model
+ * (scope 1, n = L*H); inside a set heads are ranked by descending value, equal values by ascending index,
+ * and rank r belongs to group g with floor(g n / M) <= r < floor((g+1) n / M), the grouping
+ * uncomp_assign_budgets uses.  Reading: the paper names no clustering algorithm; this equal-size
+ * rank-based grouping is used for the per-sample clusters too.
+ *   mean[l,h]       = (1/S) sum_i erank[i,l,h]  (fp64 accumulation in a fixed order, rounded to float)
+ *   group_mean[l,h] = group of head (l,h) when the set is ranked by mean
+ *   votes[l,h,g]    = number of samples whose own ranking puts head (l,h) in group g
+ *   group_vote[l,h] = arg max_g votes[l,h,g], the lowest g on a tie
+ *
+ * d_erank       in   [S, L, H] float, e.g. the d_erank output of uncomp_entropy for a batch of S samples
+ * S                  1 <= S <= 65535;  M: 1 <= M <= n;  n <= 8192 (UNCOMP_E_LIMIT beyond)
+ * d_mean        out  [L, H] float
+ * d_group_mean  out  [L, H] int32
+ * d_votes       out  [L, H, M] int32 (cleared by the call)
+ * d_group_vote  out  [L, H] int32
+ * ------------------------------------------------------------------------------------------------- */
+int uncomp_prepare_groups(uncomp_ctx *ctx, const float *d_erank, int32_t S, int32_t M, int32_t scope, float *d_mean,
+                          int32_t *d_group_mean, int32_t *d_votes, int32_t *d_group_vote, void *stream);
+
 /* Synchronise `stream`, copy the status word to *host_bits and clear it on the device.  The only call
  * that waits for the device. */
 int uncomp_status(uncomp_ctx *ctx, void *stream, uint32_t *host_bits);

@@ -82,6 +82,8 @@ def _load() -> C.CDLL:
     lib.uncomp_profile_slot_name.argtypes = [C.c_int]
     lib.uncomp_profile_read.restype = C.c_int
     lib.uncomp_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.uncomp_prepare_groups.restype = C.c_int
+    lib.uncomp_prepare_groups.argtypes = [vp, fp, C.c_int32, C.c_int32, C.c_int32, fp, i32p, i32p, i32p, vp]
     lib.uncomp_decode_update.restype = C.c_int
     lib.uncomp_decode_update.argtypes = [vp, vp, vp, vp, i32p, i64p, i32p, C.c_int32, C.c_int64, C.c_int32, C.c_float,
                                          vp, vp, i32p, fp, fp, i32p, vp]
@@ -265,6 +267,19 @@ def uncomp_decode_update(ctx: Context, qnew: torch.Tensor, knew: torch.Tensor, v
     _check(lib.uncomp_decode_update(ctx.handle, _ptr(qnew), _ptr(knew), _ptr(vnew), _ptr(new_pos), _ptr(offsets),
                                     _ptr(lens), max_cap, Kc.shape[0], protect, scale, _ptr(Kc), _ptr(Vc), _ptr(pos),
                                     _ptr(cum), _ptr(p), _ptr(evicted), _stream(stream)), "uncomp_decode_update")
+
+
+def uncomp_prepare_groups(ctx: Context, erank: torch.Tensor, M: int, scope: int = 0, stream=None):
+    """erank [S, L, H] float32 -> (mean [L, H], group_mean [L, H], votes [L, H, M], group_vote [L, H])."""
+    S, L, H = erank.shape
+    dev = erank.device
+    mean = torch.empty(L, H, dtype=torch.float32, device=dev)
+    gm = torch.empty(L, H, dtype=torch.int32, device=dev)
+    votes = torch.empty(L, H, M, dtype=torch.int32, device=dev)
+    gv = torch.empty(L, H, dtype=torch.int32, device=dev)
+    _check(lib.uncomp_prepare_groups(ctx.handle, _ptr(erank), S, M, scope, _ptr(mean), _ptr(gm), _ptr(votes), _ptr(gv),
+                                     _stream(stream)), "uncomp_prepare_groups")
+    return mean, gm, votes, gv
 
 
 def uncomp_status(ctx: Context, stream=None) -> int:

@@ -205,7 +205,8 @@ const char *uncomp_profile_slot_name(int slot) {
     static const char *names[kSlotCount] = {"gram", "eigen_entropy", "budgets", "score_stats", "stats_merge",
                                             "score_colsum", "pool_select", "compact", "gram_score_stats",
                                             "evict_logits", "evict_scores", "evict_gather",
-                                            "decode_logits", "decode_accumulate", "decode_commit"};
+                                            "decode_logits", "decode_accumulate", "decode_commit",
+                                            "prepare_vote", "prepare_finish"};
     return slot >= 0 && slot < kSlotCount ? names[slot] : "";
 }
 
@@ -404,6 +405,19 @@ int uncomp_decode_update(uncomp_ctx *ctx, const void *d_qnew, const void *d_knew
         reinterpret_cast<float *>(ctx->ws + p.off_dec_stats), ctx->ws + p.off_dec_part,
         reinterpret_cast<float *>(ctx->ws + p.off_dec_new), reinterpret_cast<uint32_t *>(ctx->ws + p.off_status),
         ctx->prof, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+int uncomp_prepare_groups(uncomp_ctx *ctx, const float *d_erank, int32_t S, int32_t M, int32_t scope, float *d_mean,
+                          int32_t *d_group_mean, int32_t *d_votes, int32_t *d_group_vote, void *stream) {
+    if (!ctx || !d_erank || !d_mean || !d_group_mean || !d_votes || !d_group_vote) return UNCOMP_E_NULL;
+    const uncomp_shape &s = ctx->plan.shape;
+    const int n = scope ? s.L * s.H : s.H;
+    if (S < 1 || M < 1 || M > n || (scope != 0 && scope != 1)) return UNCOMP_E_PARAM;
+    if (n > 8192 || S > 65535) return UNCOMP_E_LIMIT;
+    cudaError_t e = launch_prepare_groups(d_erank, S, s.L, s.H, M, scope, d_mean, d_group_mean, d_votes, d_group_vote,
+                                          ctx->prof, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;
 }

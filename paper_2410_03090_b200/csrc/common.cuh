@@ -65,7 +65,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 // Optional per-kernel timing with CUDA events on the launching stream (host objects only).
 enum Slot { kSlotGram = 0, kSlotEigen, kSlotBudgets, kSlotScoreStats, kSlotStatsMerge, kSlotScoreColsum,
             kSlotPoolSelect, kSlotCompact, kSlotGramStats, kSlotEvictLogits, kSlotEvictScores, kSlotEvictGather,
-            kSlotDecodeLogits, kSlotDecodeAccumulate, kSlotDecodeCommit, kSlotCount };
+            kSlotDecodeLogits, kSlotDecodeAccumulate, kSlotDecodeCommit, kSlotPrepareVote,
+            kSlotPrepareFinish, kSlotCount };
 enum { kScorePhaseStats = 1, kScorePhaseColsum = 2 };
 struct Profiler;
 void prof_begin(Profiler *p, int slot, cudaStream_t st);
@@ -112,6 +113,9 @@ cudaError_t launch_decode_update(const Plan &p, const void *d_q, const void *d_k
                                  int protect, float scale, void *d_Kc, void *d_Vc, int32_t *d_pos, float *d_cum,
                                  float *d_p, int32_t *d_evicted, float *d_logits, float *d_stats, void *d_partial,
                                  float *d_new_cum, uint32_t *d_status, Profiler *prof, cudaStream_t st);
+cudaError_t launch_prepare_groups(const float *d_erank, int S, int L, int H, int M, int scope, float *d_mean,
+                                  int32_t *d_group_mean, int32_t *d_votes, int32_t *d_group_vote, Profiler *prof,
+                                  cudaStream_t st);
 cudaError_t launch_compact(const Plan &p, const void *dK, const void *dV, const UnitAddr &aK, const UnitAddr &aV,
                            const int32_t *d_indices, const int64_t *d_offsets, void *dKc, void *dVc,
                            cudaStream_t st);
