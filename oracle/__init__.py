@@ -242,3 +242,19 @@ def majority_vote(erank, M: int, scope: int = 0):
     if _lib.oracle_majority_vote(_p(erank, _dp), S, L, H, int(M), int(scope), _p(votes, _i32p), _p(labels, _i32p)) != 0:
         raise ValueError("M must be between 1 and the size of the ranking set")
     return votes, labels
+
+
+def entropy_wide(X, k_trunc: int = 32, center: bool = True, norm: int = 0, return_spectrum: bool = False):
+    """(H_k, erank_k[, spectrum]) of a wide token matrix X [N, D] (hidden states, or a layer's heads side by
+    side; Section 3.1 Eq. 1 and Section 3.2).  The same definition as `entropy`, with the two heavy steps
+    handed to library routines so that D in the thousands finishes in seconds: the centred scatter matrix is a
+    library matrix product of the centred rows, its eigenvalues come from the library's symmetric
+    eigensolver; truncation and entropy are the oracle's own `truncated_entropy`."""
+    X = _f64(X)
+    if center:
+        X = X - X.mean(axis=0, keepdims=True)
+    lam = np.linalg.eigvalsh(X.T @ X)[::-1].copy()
+    H, E = truncated_entropy(lam, k_trunc, norm)
+    if return_spectrum:
+        return H, E, lam
+    return H, E
