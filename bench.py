@@ -135,6 +135,10 @@ def kernel_specs(wl, peaks, sustained: bool, D=None, n_keep=None, cache_rows=Non
         "decode_commit": ("hbm", None, None, None),
         "prepare_vote": ("alu", None, None, None),
         "prepare_finish": ("alu", None, None, None),
+        "wide_gram": ("tensor", None, None, None),
+        "wide_assemble": ("hbm", None, None, None),
+        "wide_tridiag": ("alu", None, None, None),
+        "wide_eigen_entropy": ("alu", None, None, None),
     }
 
 

@@ -334,6 +334,31 @@ int uncomp_decode_update(uncomp_ctx *ctx, const void *d_qnew, const void *d_knew
 int uncomp_prepare_groups(uncomp_ctx *ctx, const float *d_erank, int32_t S, int32_t M, int32_t scope, float *d_mean,
                           int32_t *d_group_mean, int32_t *d_votes, int32_t *d_group_vote, void *stream);
 
+/* ---------------------------------------------------------------------------------------------------
+ * uncomp_entropy_wide -- Section 3.1 Eq. 1 for token vectors x_i in R^D with D beyond a head (the hidden
+ * states of a layer, D = 4096, or the heads of a layer side by side), Lemma 2 and Section 3.2: the same
+ * H_k and erank_k as uncomp_entropy, of `count` matrices X_i [N, D] (bf16; the context must be a bf16
+ * one).  The D x D scatter matrix is formed on the tensor cores, tridiagonalised in fp32 by one
+ * cooperative kernel that spans the GPU and its k largest eigenvalues are found in fp64 (Sturm counts).
+ *
+ * d_X            in   matrix i starts at element i * stride_matrix; token rows stride_row elements apart
+ *                     (stride_row >= D, both strides multiples of 8 elements), features contiguous
+ * N, D                N >= 2; 128 <= D <= 4096 (UNCOMP_E_LIMIT beyond), D a multiple of 64
+ * params              as for uncomp_entropy, k_trunc <= 256
+ * d_scratch           caller-owned device memory, 256-byte aligned, at least
+ *                     uncomp_entropy_wide_scratch_bytes(N, D) bytes (0 for an unsupported shape); the
+ *                     matrices are processed one after the other and share it
+ * d_entropy      out  [count] float;  d_erank out [count] float, may be NULL
+ * d_spectrum     out  [count, min(k_trunc, D)] double, the largest eigenvalues, descending; may be NULL
+ * The cooperative kernel needs the GPU to itself while it runs: launching it on a device whose SMs are
+ * held by another long-running kernel delays it, it never deadlocks (its grid barrier gives up after a
+ * bounded number of polls and raises UNCOMP_STATUS_TIMEOUT).
+ * ------------------------------------------------------------------------------------------------- */
+size_t uncomp_entropy_wide_scratch_bytes(int32_t N, int32_t D);
+int uncomp_entropy_wide(uncomp_ctx *ctx, const void *d_X, int32_t count, int64_t stride_matrix, int64_t stride_row,
+                        int32_t N, int32_t D, const uncomp_entropy_params *params, void *d_scratch, size_t scratch_bytes,
+                        float *d_entropy, float *d_erank, double *d_spectrum, void *stream);
+
 /* Synchronise `stream`, copy the status word to *host_bits and clear it on the device.  The only call
  * that waits for the device. */
 int uncomp_status(uncomp_ctx *ctx, void *stream, uint32_t *host_bits);

@@ -82,6 +82,11 @@ def _load() -> C.CDLL:
     lib.uncomp_profile_slot_name.argtypes = [C.c_int]
     lib.uncomp_profile_read.restype = C.c_int
     lib.uncomp_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.uncomp_entropy_wide_scratch_bytes.restype = C.c_size_t
+    lib.uncomp_entropy_wide_scratch_bytes.argtypes = [C.c_int32, C.c_int32]
+    lib.uncomp_entropy_wide.restype = C.c_int
+    lib.uncomp_entropy_wide.argtypes = [vp, vp, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
+                                        C.POINTER(uncomp_entropy_params), vp, C.c_size_t, fp, fp, dp, vp]
     lib.uncomp_prepare_groups.restype = C.c_int
     lib.uncomp_prepare_groups.argtypes = [vp, fp, C.c_int32, C.c_int32, C.c_int32, fp, i32p, i32p, i32p, vp]
     lib.uncomp_decode_update.restype = C.c_int
@@ -267,6 +272,26 @@ def uncomp_decode_update(ctx: Context, qnew: torch.Tensor, knew: torch.Tensor, v
     _check(lib.uncomp_decode_update(ctx.handle, _ptr(qnew), _ptr(knew), _ptr(vnew), _ptr(new_pos), _ptr(offsets),
                                     _ptr(lens), max_cap, Kc.shape[0], protect, scale, _ptr(Kc), _ptr(Vc), _ptr(pos),
                                     _ptr(cum), _ptr(p), _ptr(evicted), _stream(stream)), "uncomp_decode_update")
+
+
+def uncomp_entropy_wide(ctx: Context, X: torch.Tensor, k_trunc: int = 32, center: int = 1, norm: int = 0,
+                        max_iters: int = 0, scratch: Optional[torch.Tensor] = None, spectrum: bool = False, stream=None):
+    """X [count, N, D] bf16 (rows may be strided, features contiguous) -> (entropy [count], erank [count]
+    [, spectrum [count, k]])."""
+    if X.dim() != 3 or X.stride(2) != 1:
+        raise ValueError("expected X [count, N, D] with a contiguous last dimension")
+    count, N, D = X.shape
+    need = lib.uncomp_entropy_wide_scratch_bytes(N, D)
+    if scratch is None:
+        scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=X.device)
+    ent = torch.empty(count, dtype=torch.float32, device=X.device)
+    er = torch.empty(count, dtype=torch.float32, device=X.device)
+    spec = torch.empty(count, min(k_trunc, D), dtype=torch.float64, device=X.device) if spectrum else None
+    params = uncomp_entropy_params(k_trunc, center, norm, max_iters)
+    _check(lib.uncomp_entropy_wide(ctx.handle, _ptr(X), count, X.stride(0), X.stride(1), N, D, C.byref(params),
+                                   _ptr(scratch), scratch.numel(), _ptr(ent), _ptr(er), _ptr(spec), _stream(stream)),
+           "uncomp_entropy_wide")
+    return (ent, er, spec) if spectrum else (ent, er)
 
 
 def uncomp_prepare_groups(ctx: Context, erank: torch.Tensor, M: int, scope: int = 0, stream=None):

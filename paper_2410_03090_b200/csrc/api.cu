@@ -206,7 +206,8 @@ const char *uncomp_profile_slot_name(int slot) {
                                             "score_colsum", "pool_select", "compact", "gram_score_stats",
                                             "evict_logits", "evict_scores", "evict_gather",
                                             "decode_logits", "decode_accumulate", "decode_commit",
-                                            "prepare_vote", "prepare_finish"};
+                                            "prepare_vote", "prepare_finish",
+                                            "wide_gram", "wide_assemble", "wide_tridiag", "wide_eigen_entropy"};
     return slot >= 0 && slot < kSlotCount ? names[slot] : "";
 }
 
@@ -419,6 +420,38 @@ int uncomp_prepare_groups(uncomp_ctx *ctx, const float *d_erank, int32_t S, int3
     cudaError_t e = launch_prepare_groups(d_erank, S, s.L, s.H, M, scope, d_mean, d_group_mean, d_votes, d_group_vote,
                                           ctx->prof, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
+size_t uncomp_entropy_wide_scratch_bytes(int32_t N, int32_t D) {
+    if (N < 2 || D < 128 || D > 4096 || D % 64 != 0) return 0;
+    return entropy_wide_scratch_bytes(N, D);
+}
+
+int uncomp_entropy_wide(uncomp_ctx *ctx, const void *d_X, int32_t count, int64_t stride_matrix, int64_t stride_row,
+                        int32_t N, int32_t D, const uncomp_entropy_params *params, void *d_scratch, size_t scratch_bytes,
+                        float *d_entropy, float *d_erank, double *d_spectrum, void *stream) {
+    if (!ctx || !d_X || !params || !d_scratch || !d_entropy) return UNCOMP_E_NULL;
+    if (ctx->plan.shape.dtype != UNCOMP_BF16) return UNCOMP_E_SHAPE;
+    if (count < 1 || N < 2 || D < 128 || D % 64 != 0) return UNCOMP_E_SHAPE;
+    if (D > 4096) return UNCOMP_E_LIMIT;
+    if (!aligned16(d_X) || !aligned16(d_scratch) || ((uintptr_t)d_scratch & 255) != 0 || stride_row < D ||
+        stride_row % 8 != 0 || stride_matrix % 8 != 0)
+        return UNCOMP_E_ALIGN;
+    if (params->k_trunc < 1 || params->k_trunc > 256 || (params->center != 0 && params->center != 1) ||
+        (params->norm != 0 && params->norm != 1) || params->max_iters < 0)
+        return UNCOMP_E_PARAM;
+    if (scratch_bytes < entropy_wide_scratch_bytes(N, D)) return UNCOMP_E_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int k = params->k_trunc < D ? params->k_trunc : D;
+    for (int i = 0; i < count; ++i) {
+        const unsigned char *Xi = static_cast<const unsigned char *>(d_X) + (size_t)i * stride_matrix * 2;
+        cudaError_t e = launch_entropy_wide(Xi, stride_row, N, D, *params, static_cast<unsigned char *>(d_scratch),
+                                            d_entropy + i, d_erank ? d_erank + i : nullptr,
+                                            d_spectrum ? d_spectrum + (size_t)i * k : nullptr,
+                                            reinterpret_cast<uint32_t *>(ctx->ws + ctx->plan.off_status), ctx->prof, st);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
     return UNCOMP_OK;
 }
 

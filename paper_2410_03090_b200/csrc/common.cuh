@@ -66,7 +66,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 enum Slot { kSlotGram = 0, kSlotEigen, kSlotBudgets, kSlotScoreStats, kSlotStatsMerge, kSlotScoreColsum,
             kSlotPoolSelect, kSlotCompact, kSlotGramStats, kSlotEvictLogits, kSlotEvictScores, kSlotEvictGather,
             kSlotDecodeLogits, kSlotDecodeAccumulate, kSlotDecodeCommit, kSlotPrepareVote,
-            kSlotPrepareFinish, kSlotCount };
+            kSlotPrepareFinish, kSlotWideGram, kSlotWideAssemble, kSlotWideTridiag, kSlotWideSturm, kSlotCount };
 enum { kScorePhaseStats = 1, kScorePhaseColsum = 2 };
 struct Profiler;
 void prof_begin(Profiler *p, int slot, cudaStream_t st);
@@ -116,6 +116,10 @@ cudaError_t launch_decode_update(const Plan &p, const void *d_q, const void *d_k
 cudaError_t launch_prepare_groups(const float *d_erank, int S, int L, int H, int M, int scope, float *d_mean,
                                   int32_t *d_group_mean, int32_t *d_votes, int32_t *d_group_vote, Profiler *prof,
                                   cudaStream_t st);
+size_t entropy_wide_scratch_bytes(int N, int D);
+cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const uncomp_entropy_params &ep,
+                                unsigned char *scratch, float *d_entropy, float *d_erank, double *d_spectrum,
+                                uint32_t *d_status, Profiler *prof, cudaStream_t st);
 cudaError_t launch_compact(const Plan &p, const void *dK, const void *dV, const UnitAddr &aK, const UnitAddr &aV,
                            const int32_t *d_indices, const int64_t *d_offsets, void *dKc, void *dVc,
                            cudaStream_t st);

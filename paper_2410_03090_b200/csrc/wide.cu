@@ -1,0 +1,533 @@
+// Truncated matrix entropy of WIDE token matrices X [N, D], D up to 4096: hidden states, or the heads of a
+// layer side by side (paper Section 3.1 Eq. 1 with x_i in R^D, Lemma 2, Section 3.2; the appendix section on
+// the truncated effective rank of hidden states).  The D x D scatter matrix does not fit an SM, so the stage
+// is split differently from the per-head path:
+//   1. column sums       s = X^T 1, fp64, token chunks summed in a fixed order;
+//   2. Gram              G = X^T X on tcgen05: a CTA owns a 256 x 256 block pair (I <= J) of G and a token
+//                        chunk; per 64-token stage TMA brings the 256 features of block I and of block J
+//                        (64-feature boxes, 128B swizzle); both MMA operands are read MN-major, two
+//                        M = 128, N = 256 accumulators fill the 512 TMEM columns; partial blocks to scratch;
+//   3. assemble          C = G - s s^T / N (fp64 subtraction), stored as a full symmetric fp32 matrix;
+//   4. tridiagonalise    Householder on the whole GPU: one cooperative launch, rows of the trailing matrix
+//                        spread over all warps, ONE grid barrier per column.  The rank-2 update of column k
+//                        is applied while the matrix is swept for the matrix-vector product of column k + 1,
+//                        so the matrix (64 MB at D = 4096, resident in L2) is read and written once per column;
+//   5. eigenvalues       Sturm-count multi-section (fp64) for the k largest of the tridiagonal matrix, then
+//                        H_k and erank_k.
+// Every wait is bounded: the TMA / MMA barriers as in the other tensor-core kernels, the grid barrier by a
+// poll limit after which the kernel raises UNCOMP_STATUS_TIMEOUT and all CTAs leave.
+#include <math.h>
+
+#include "tc_common.cuh"
+
+namespace uncomp {
+
+namespace {
+// ------------------------------------------------------------------------------------------ 1. column sums
+constexpr int kColChunks = 32;
+
+__global__ void __launch_bounds__(256) wide_colsum_kernel(const __nv_bfloat16 *__restrict__ X, int64_t sN, int N, int D,
+                                                         double *__restrict__ part) {
+    const int f = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y;
+    if (f >= D) return;
+    const int per = (N + kColChunks - 1) / kColChunks;
+    const int t0 = c * per, t1 = min(N, t0 + per);
+    double acc = 0.0;
+    for (int t = t0; t < t1; ++t) acc += (double)__bfloat162float(X[(int64_t)t * sN + f]);
+    part[(size_t)c * D + f] = acc;
+}
+
+__global__ void __launch_bounds__(256) wide_colsum_reduce_kernel(const double *__restrict__ part, int D,
+                                                                double *__restrict__ s) {
+    const int f = blockIdx.x * 256 + threadIdx.x;
+    if (f >= D) return;
+    double acc = 0.0;
+    for (int c = 0; c < kColChunks; ++c) acc += part[(size_t)c * D + f];
+    s[f] = acc;
+}
+
+// ------------------------------------------------------------------------------------------------ 2. Gram
+constexpr int kWTok = 64;                        // tokens per stage
+constexpr int kWRegion = 64 * 128;               // 8 KB: 64 tokens x 64 features (128 B rows)
+constexpr int kWHalf = 4 * kWRegion;             // 32 KB: the 256 features of one block
+constexpr int kWStage = 2 * kWHalf;              // 64 KB: block I then block J
+constexpr int kWStages = 3;
+constexpr int kWThreads = 192;
+constexpr int kWBlock = 256;                     // features per block of G
+
+struct WideTail {
+    uint64_t full[kWStages];
+    uint64_t empty[kWStages];
+    uint64_t accum;
+    uint32_t tmem_base;
+    uint32_t abort;
+};
+constexpr int kWSmem = 1024 + kWStages * kWStage + (int)sizeof(WideTail);
+
+// grid (block pairs, token chunks)
+__global__ void __launch_bounds__(kWThreads, 1)
+gram_wide_kernel(const __grid_constant__ CUtensorMap tmap, int N, int nblk, int chunk, float *__restrict__ partials,
+                 uint32_t *__restrict__ status) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw_addr = tc::smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    unsigned char *smem = smem_raw + pad;
+    const uint32_t tiles_addr = raw_addr + pad;
+    WideTail &T = *reinterpret_cast<WideTail *>(smem + kWStages * kWStage);
+
+    int I = 0, J = 0;
+    {
+        int rem = blockIdx.x;
+        for (I = 0; I < nblk; ++I) {
+            const int cnt = nblk - I;
+            if (rem < cnt) { J = I + rem; break; }
+            rem -= cnt;
+        }
+    }
+    const bool diag = I == J;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t0 = blockIdx.y * chunk, t1 = min(N, t0 + chunk);
+    const int ntiles = (t1 - t0 + kWTok - 1) / kWTok;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kWStages; ++s) {
+            tc::mbar_init(tc::smem_u32(&T.full[s]), 1);
+            tc::mbar_init(tc::smem_u32(&T.empty[s]), 1);
+        }
+        tc::mbar_init(tc::smem_u32(&T.accum), 1);
+        T.abort = 0;
+        tc::fence_mbar_init();
+    }
+    if (warp == 5) {
+        tc::tmem_alloc(tc::smem_u32(&T.tmem_base), 512);
+        tc::tmem_relinquish();
+    }
+    if (warp == 4 && lane == 0) tc::prefetch_tmap(&tmap);
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem = T.tmem_base;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int i = 0; i < ntiles; ++i, ++issued) {
+                const int s = i % kWStages;
+                if (i >= kWStages && !tc::mbar_wait(tc::smem_u32(&T.empty[s]), ((i / kWStages) - 1) & 1, status)) {
+                    T.abort = 1;
+                    break;
+                }
+                const uint32_t bar = tc::smem_u32(&T.full[s]);
+                const uint32_t dst = tiles_addr + s * kWStage;
+                tc::mbar_expect_tx(bar, diag ? kWHalf : kWStage);
+#pragma unroll
+                for (int r = 0; r < 4; ++r) tc::tma_load_3d(dst + r * kWRegion, &tmap, bar, I * kWBlock + r * 64, t0 + i * kWTok, 0);
+                if (!diag) {
+#pragma unroll
+                    for (int r = 0; r < 4; ++r)
+                        tc::tma_load_3d(dst + kWHalf + r * kWRegion, &tmap, bar, J * kWBlock + r * 64, t0 + i * kWTok, 0);
+                }
+            }
+            if (T.abort) {
+                for (int i = max(0, issued - kWStages); i < issued; ++i)
+                    tc::mbar_wait(tc::smem_u32(&T.full[i % kWStages]), (i / kWStages) & 1, status);
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = tc::idesc_bf16_f32(128, 256, 1, 1);
+            // MN-major, 128-byte swizzle: 64-feature regions kWRegion apart (LBO), 8-token groups 1024 B apart
+            // (SBO); 16 tokens further = 2048 B = +128 in the 16-byte address field
+            const uint64_t base_desc = tc::smem_desc_sw128(tiles_addr, kWRegion, 1024);
+            const uint32_t dhi = tc::desc_hi(base_desc);
+            bool ok = true;
+            for (int i = 0; i < ntiles && ok; ++i) {
+                const int s = i % kWStages;
+                ok = tc::mbar_wait(tc::smem_u32(&T.full[s]), (i / kWStages) & 1, status);
+                if (!ok) { T.abort = 1; break; }
+                tc::tc_fence_after();
+                const uint32_t lo = tc::desc_lo(base_desc) + (uint32_t)(s * (kWStage >> 4));
+                const uint32_t b_lo = lo + (diag ? 0u : (uint32_t)(kWHalf >> 4));
+#pragma unroll
+                for (int k = 0; k < kWTok / 16; ++k) {
+                    const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
+                    tc::mma_f16_ss_lohi(tmem, lo + k * 128, b_lo + k * 128, dhi, idesc, acc);
+                    tc::mma_f16_ss_lohi(tmem + 256, lo + (uint32_t)((2 * kWRegion) >> 4) + k * 128, b_lo + k * 128, dhi, idesc,
+                                        acc);
+                }
+                tc::mma_commit(tc::smem_u32(&T.empty[s]));
+            }
+            tc::mma_commit(tc::smem_u32(&T.accum));
+        }
+    } else {
+        const bool ok = tc::mbar_wait(tc::smem_u32(&T.accum), 0, status);
+        tc::tc_fence_after();
+        if (ok && !T.abort) {
+            const int m = warp * 32 + lane;
+            uint32_t r[32];
+#pragma unroll 1
+            for (int mi = 0; mi < 2; ++mi) {
+                float *out = partials + (((size_t)blockIdx.y * gridDim.x + blockIdx.x) * 2 + mi) * (128 * kWBlock) +
+                             (size_t)m * kWBlock;
+#pragma unroll 1
+                for (int c0 = 0; c0 < kWBlock; c0 += 32) {
+                    tc::tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + mi * 256 + c0, r);
+                    tc::tmem_ld_wait();
+                    float4 *dst = reinterpret_cast<float4 *>(out + c0);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                             __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+                }
+            }
+        }
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 5) tc::tmem_dealloc(tmem, 512);
+}
+
+// -------------------------------------------------------------------------------------------- 3. assemble
+// grid (block pairs, 256 rows of the pair's block), thread = column.  Only the upper triangle of a diagonal
+// block is taken from the MMA result and mirrored, so C is symmetric bit for bit.
+__global__ void __launch_bounds__(256) wide_assemble_kernel(const float *__restrict__ partials, int pairs, int chunks,
+                                                           int nblk, int D, int N, int center,
+                                                           const double *__restrict__ s, float *__restrict__ C) {
+    int I = 0, J = 0;
+    {
+        int rem = blockIdx.x;
+        for (I = 0; I < nblk; ++I) {
+            const int cnt = nblk - I;
+            if (rem < cnt) { J = I + rem; break; }
+            rem -= cnt;
+        }
+    }
+    const int r = blockIdx.y, c = threadIdx.x;
+    const int gi = I * kWBlock + r, gj = J * kWBlock + c;
+    if (gi >= D || gj >= D || (I == J && r > c)) return;
+    const int mi = r >> 7, m = r & 127;
+    double acc = 0.0;
+    for (int ch = 0; ch < chunks; ++ch)
+        acc += (double)partials[(((size_t)ch * pairs + blockIdx.x) * 2 + mi) * (128 * kWBlock) + (size_t)m * kWBlock + c];
+    if (center) acc -= s[gi] * s[gj] / (double)N;
+    const float v = (float)acc;
+    C[(size_t)gi * D + gj] = v;
+    C[(size_t)gj * D + gi] = v;
+}
+
+// ------------------------------------------------------------------------------------- 4. tridiagonalisation
+constexpr int kTriThreads = 512;
+constexpr int kTriWarps = kTriThreads / 32;
+constexpr unsigned kBarrierSpin = 1u << 22;
+
+__device__ __forceinline__ float tri_block_sum(float v, float *red) {
+    v = warp_sum(v);
+    __syncthreads();                 // red is free again
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < kTriWarps; ++i) t += red[i];
+    return t;
+}
+
+// All CTAs of a cooperative launch meet here.  `bar` counts arrivals monotonically.
+__device__ __forceinline__ bool tri_grid_barrier(unsigned *bar, unsigned &phase, uint32_t *status, int *flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(bar, 1u);
+        const unsigned target = (phase + 1u) * gridDim.x;
+        bool ok = false;
+        for (unsigned it = 0; it < kBarrierSpin; ++it) {
+            unsigned cur;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(cur) : "l"(bar) : "memory");
+            if (cur >= target) { ok = true; break; }
+        }
+        if (!ok) atomicOr(status, (uint32_t)UNCOMP_STATUS_TIMEOUT);
+        *flag = ok ? 1 : 0;
+    }
+    __syncthreads();
+    ++phase;
+    return *flag != 0;
+}
+
+// A: full symmetric fp32 matrix [D, D], destroyed.  Output: diagonal a[D] and off-diagonal e[D - 1].
+// State at the top of iteration k: rows >= k of A hold the matrix after the reflections of columns 0 .. k - 2;
+// the rank-2 update of column k - 1, A -= 2 (v w^T + w v^T) on rows and columns >= k, is still pending and kept
+// as (v, w) in shared memory by every CTA.
+__global__ void __launch_bounds__(kTriThreads, 1) tridiag_wide_kernel(float *__restrict__ A, int D, double *__restrict__ a_out,
+                                                                     double *__restrict__ e_out, float *__restrict__ pbuf,
+                                                                     unsigned *bar, uint32_t *__restrict__ status) {
+    extern __shared__ float sm[];
+    float *v = sm, *w = sm + D, *vn = sm + 2 * D;
+    __shared__ float red[kTriWarps];
+    __shared__ int flag;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int total_warps = gridDim.x * kTriWarps, gw = blockIdx.x * kTriWarps + warp;
+    for (int i = tid; i < D; i += kTriThreads) { v[i] = 0.f; w[i] = 0.f; }
+    __syncthreads();
+    unsigned phase = 0;
+    for (int k = 0; k + 2 < D; ++k) {
+        // row k with the pending update applied: diagonal entry and the column to eliminate
+        const float vk = v[k], wk = w[k];
+        for (int j = k + tid; j < D; j += kTriThreads)
+            vn[j] = __ldcg(A + (size_t)k * D + j) - 2.f * (vk * w[j] + wk * v[j]);
+        __syncthreads();
+        float part = 0.f;
+        for (int j = k + 1 + tid; j < D; j += kTriThreads) part += vn[j] * vn[j];
+        const float sigma = tri_block_sum(part, red);
+        const float akk = vn[k], x0 = vn[k + 1];
+        float alpha = 0.f, inv = 0.f;
+        if (sigma > 0.f) {
+            alpha = -copysignf(sqrtf(sigma), x0);
+            inv = 1.f / sqrtf(2.f * (sigma - alpha * x0));     // 1 / |x - alpha e_1|
+        }
+        __syncthreads();                                       // every thread has read vn[k], vn[k + 1]
+        for (int j = k + 1 + tid; j < D; j += kTriThreads) vn[j] = (vn[j] - (j == k + 1 ? alpha : 0.f)) * inv;
+        if (blockIdx.x == 0 && tid == 0) { a_out[k] = (double)akk; e_out[k] = (double)alpha; }
+        __syncthreads();
+        // sweep: apply the pending update to rows >= k + 1 and form p = A' vn on the fly
+        float *pw = pbuf + (size_t)(k & 1) * D;
+        for (int i = k + 1 + gw; i < D; i += total_warps) {
+            const float vi = v[i], wi = w[i];
+            float *row = A + (size_t)i * D;
+            float acc = 0.f;
+            for (int j = k + 1 + lane; j < D; j += 32) {
+                const float x = __ldcg(row + j) - 2.f * (vi * w[j] + wi * v[j]);
+                __stcg(row + j, x);
+                acc = fmaf(x, vn[j], acc);
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) __stcg(pw + i, acc);
+        }
+        if (!tri_grid_barrier(bar, phase, status, &flag)) return;
+        // new pending update: w = p - (vn . p) vn, v = vn
+        part = 0.f;
+        for (int j = k + 1 + tid; j < D; j += kTriThreads) {
+            const float pj = __ldcg(pw + j);
+            w[j] = pj;
+            part += vn[j] * pj;
+        }
+        const float Kdot = tri_block_sum(part, red);
+        for (int j = k + 1 + tid; j < D; j += kTriThreads) {
+            w[j] -= Kdot * vn[j];
+            v[j] = vn[j];
+        }
+        __syncthreads();
+    }
+    if (blockIdx.x == 0 && tid == 0) {
+        const int i = D - 2, j = D - 1;
+        a_out[i] = (double)(__ldcg(A + (size_t)i * D + i) - 4.f * v[i] * w[i]);
+        e_out[i] = (double)(__ldcg(A + (size_t)i * D + j) - 2.f * (v[i] * w[j] + w[i] * v[j]));
+        a_out[j] = (double)(__ldcg(A + (size_t)j * D + j) - 4.f * v[j] * w[j]);
+    }
+}
+
+// --------------------------------------------------------------------------------- 5. eigenvalues, entropy
+constexpr int kSturmThreads = 256;
+constexpr int kSturmMaxK = 256;
+
+// number of eigenvalues of the tridiagonal matrix (a, e) below x
+__device__ int sturm_count_wide(const double *__restrict__ a, const double *__restrict__ e, int D, double x, double tiny) {
+    double q = a[0] - x;
+    if (fabs(q) < tiny) q = -tiny;
+    int cnt = q < 0.0;
+    for (int i = 1; i < D; ++i) {
+        const double ei = e[i - 1];
+        q = (a[i] - x) - ei * ei / q;
+        if (fabs(q) < tiny) q = -tiny;
+        cnt += q < 0.0;
+    }
+    return cnt;
+}
+
+__global__ void __launch_bounds__(kSturmThreads) sturm_wide_kernel(const double *__restrict__ a, const double *__restrict__ e,
+                                                                  int D, int k, int norm, int max_iters,
+                                                                  float *__restrict__ H_out, float *__restrict__ erank_out,
+                                                                  double *__restrict__ spectrum,
+                                                                  uint32_t *__restrict__ status) {
+    __shared__ double redlo[kSturmThreads / 32], redhi[kSturmThreads / 32], redtr[kSturmThreads / 32];
+    __shared__ double xs[kSturmThreads];
+    __shared__ int cs[kSturmThreads];
+    __shared__ double lam[kSturmMaxK];
+    __shared__ double bounds[3];
+    __shared__ int not_conv;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    // Gershgorin interval and trace
+    double lo = 1e300, hi = -1e300, tr = 0.0;
+    for (int i = tid; i < D; i += kSturmThreads) {
+        const double r = (i > 0 ? fabs(e[i - 1]) : 0.0) + (i + 1 < D ? fabs(e[i]) : 0.0);
+        lo = fmin(lo, a[i] - r);
+        hi = fmax(hi, a[i] + r);
+        tr += a[i];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fmin(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmax(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+        tr += __shfl_xor_sync(0xffffffffu, tr, o);
+    }
+    if (lane == 0) { redlo[wid] = lo; redhi[wid] = hi; redtr[wid] = tr; }
+    if (tid == 0) not_conv = 0;
+    __syncthreads();
+    if (tid == 0) {
+        double l = redlo[0], h = redhi[0], t = 0.0;
+        for (int i = 0; i < kSturmThreads / 32; ++i) { l = fmin(l, redlo[i]); h = fmax(h, redhi[i]); t += redtr[i]; }
+        const double span = fmax(h - l, 1e-300);
+        bounds[0] = l - 1e-9 * span;
+        bounds[1] = h + 1e-9 * span;
+        bounds[2] = t;
+    }
+    __syncthreads();
+    lo = bounds[0];
+    hi = bounds[1];
+    const double radius = fmax(fabs(lo), fabs(hi));
+    const double tiny = fmax(radius, 1e-280) * 1e-19;      // floor of a pivot of the Sturm recurrence
+    const double tol = radius * 1e-13;
+    // coarse round: 256 points over the interval
+    xs[tid] = lo + (hi - lo) * (double)tid / (double)(kSturmThreads - 1);
+    cs[tid] = sturm_count_wide(a, e, D, xs[tid], tiny);
+    __syncthreads();
+    // teams of 8 lanes refine one eigenvalue each; target t (0 = largest) is ascending index D - 1 - t
+    const int team = tid >> 3, tl = tid & 7, teams = kSturmThreads / 8;
+    const int rounds = max_iters > 0 ? max_iters : 16;
+    for (int t = team; t < k; t += teams) {
+        const int m = D - 1 - t;
+        // bracket from the coarse round: count(xl) <= m < count(xh)
+        int p = 0;
+        for (int s = 0; s < kSturmThreads; ++s)
+            if (cs[s] <= m) p = s;
+        double xl = xs[p], xh = p + 1 < kSturmThreads ? xs[p + 1] : hi;
+        int it = 0;
+        for (; it < rounds && (xh - xl) > tol; ++it) {
+            const double x = xl + (xh - xl) * (double)(tl + 1) / 9.0;
+            const int c = sturm_count_wide(a, e, D, x, tiny);
+            // lanes whose point still has count <= m form a prefix of the team
+            const unsigned shift = (unsigned)(lane & ~7);
+            const unsigned below = (__ballot_sync(0xffu << shift, c <= m) >> shift) & 0xffu;
+            const int nb = __popc(below);
+            const double step = (xh - xl) / 9.0;
+            const double nl = xl + step * (double)nb, nh = nb < 8 ? xl + step * (double)(nb + 1) : xh;
+            xl = nl;
+            xh = nh;
+        }
+        if (tl == 0) {
+            lam[t] = 0.5 * (xl + xh);
+            if ((xh - xl) > tol) not_conv = 1;
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        if (not_conv) atomicOr(status, (uint32_t)UNCOMP_STATUS_NOT_CONVERGED);
+        double denom = 0.0;
+        if (norm == 0) {
+            for (int i = 0; i < k; ++i) denom += fmax(lam[i], 0.0);
+        } else {
+            denom = bounds[2];
+        }
+        double h = 0.0;
+        for (int i = 0; i < k; ++i) {
+            const double pi = denom > 0.0 ? fmax(lam[i], 0.0) / denom : 0.0;
+            if (pi > 0.0) h -= pi * log(pi);
+        }
+        *H_out = (float)h;
+        if (erank_out) *erank_out = (float)exp(h);
+        if (spectrum)
+            for (int i = 0; i < k; ++i) spectrum[i] = lam[i];
+    }
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct WideLayout {
+    int nblk, pairs, chunk, chunks;
+    size_t off_bar, off_s, off_colpart, off_a, off_e, off_p, off_C, off_part, bytes;
+};
+
+WideLayout wide_layout(int N, int D) {
+    WideLayout w;
+    w.nblk = (D + kWBlock - 1) / kWBlock;
+    w.pairs = w.nblk * (w.nblk + 1) / 2;
+    int chunks = (2 * 148 + w.pairs - 1) / w.pairs;          // about two CTAs' worth of work per SM
+    const int max_chunks = (N + 511) / 512;
+    if (chunks > max_chunks) chunks = max_chunks;
+    if (chunks < 1) chunks = 1;
+    w.chunk = (((N + chunks - 1) / chunks) + kWTok - 1) / kWTok * kWTok;
+    w.chunks = (N + w.chunk - 1) / w.chunk;
+    size_t o = 0;
+    w.off_bar = o;      o = align256(o + 256);
+    w.off_s = o;        o = align256(o + (size_t)D * sizeof(double));
+    w.off_colpart = o;  o = align256(o + (size_t)kColChunks * D * sizeof(double));
+    w.off_a = o;        o = align256(o + (size_t)D * sizeof(double));
+    w.off_e = o;        o = align256(o + (size_t)D * sizeof(double));
+    w.off_p = o;        o = align256(o + (size_t)2 * D * sizeof(float));
+    w.off_C = o;        o = align256(o + (size_t)D * D * sizeof(float));
+    w.off_part = o;     o = align256(o + (size_t)w.chunks * w.pairs * 2 * 128 * kWBlock * sizeof(float));
+    w.bytes = o;
+    return w;
+}
+}  // namespace
+
+size_t entropy_wide_scratch_bytes(int N, int D) { return wide_layout(N, D).bytes; }
+
+cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const uncomp_entropy_params &ep,
+                                unsigned char *scratch, float *d_entropy, float *d_erank, double *d_spectrum,
+                                uint32_t *d_status, Profiler *prof, cudaStream_t st) {
+    const WideLayout w = wide_layout(N, D);
+    const __nv_bfloat16 *X = (const __nv_bfloat16 *)d_X;
+    double *s = (double *)(scratch + w.off_s), *colpart = (double *)(scratch + w.off_colpart);
+    double *a = (double *)(scratch + w.off_a), *e = (double *)(scratch + w.off_e);
+    float *pbuf = (float *)(scratch + w.off_p), *C = (float *)(scratch + w.off_C), *part = (float *)(scratch + w.off_part);
+    unsigned *bar = (unsigned *)(scratch + w.off_bar);
+    cudaError_t err = cudaMemsetAsync(bar, 0, 256, st);
+    if (err != cudaSuccess) return err;
+    {
+        ProfScope ps(prof, kSlotWideGram, st);
+        wide_colsum_kernel<<<dim3((D + 255) / 256, kColChunks), 256, 0, st>>>(X, sN, N, D, colpart);
+        wide_colsum_reduce_kernel<<<(D + 255) / 256, 256, 0, st>>>(colpart, D, s);
+        CUtensorMap tmap;
+        uint64_t dims[3] = {(uint64_t)D, (uint64_t)N, 1};
+        uint64_t str[2] = {(uint64_t)sN * 2, (uint64_t)sN * 2 * (uint64_t)N};
+        uint32_t box[3] = {64, (uint32_t)kWTok, 1};
+        err = encode_tensor_map(&tmap, d_X, 3, dims, str, box, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (err != cudaSuccess) return err;
+        err = cudaFuncSetAttribute(gram_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem);
+        if (err != cudaSuccess) return err;
+        gram_wide_kernel<<<dim3(w.pairs, w.chunks), kWThreads, kWSmem, st>>>(tmap, N, w.nblk, w.chunk, part, d_status);
+    }
+    {
+        ProfScope ps(prof, kSlotWideAssemble, st);
+        wide_assemble_kernel<<<dim3(w.pairs, kWBlock), 256, 0, st>>>(part, w.pairs, w.chunks, w.nblk, D, N, ep.center, s, C);
+    }
+    err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    {
+        ProfScope ps(prof, kSlotWideTridiag, st);
+        int dev = 0, sms = 0, per_sm = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const size_t smem = (size_t)3 * D * sizeof(float);
+        err = cudaFuncSetAttribute(tridiag_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tridiag_wide_kernel, kTriThreads, smem);
+        if (err != cudaSuccess) return err;
+        if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+        int grid = sms;                                          // one CTA per SM: all of them are resident
+        const int rows_warps = (D + kTriWarps - 1) / kTriWarps;  // no more CTAs than there are rows to share
+        if (grid > rows_warps) grid = rows_warps;
+        int Di = D;
+        void *args[] = {(void *)&C, (void *)&Di, (void *)&a, (void *)&e, (void *)&pbuf, (void *)&bar, (void *)&d_status};
+        err = cudaLaunchCooperativeKernel((const void *)tridiag_wide_kernel, dim3(grid), dim3(kTriThreads), args, smem, st);
+        if (err != cudaSuccess) return err;
+    }
+    {
+        ProfScope ps(prof, kSlotWideSturm, st);
+        const int k = ep.k_trunc < D ? ep.k_trunc : D;
+        sturm_wide_kernel<<<1, kSturmThreads, 0, st>>>(a, e, D, k, ep.norm, ep.max_iters, d_entropy, d_erank, d_spectrum,
+                                                       d_status);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace uncomp
