@@ -617,6 +617,114 @@ def run_prepare(args):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------- wide-matrix entropy
+def run_wide(args):
+    """Truncated entropy of hidden-state matrices [N, D] (paper Section 3.1 Eq. 1 with D = 4096, Section 3.2): a step
+    is the entropy of `--wide-count` matrices (the hidden states of that many layers).  Single GPU."""
+    import numpy as np
+    import torch
+    from paper_2410_03090_b200 import binding as ub
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pass has no CPU path")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    peaks = _peaks()
+    N, D, count, k = args.wide_N, args.hidden_width, args.wide_count, 32
+    g = torch.Generator(device=dev).manual_seed(11)
+    # hidden states: a few hundred strong directions with a decaying spectrum plus isotropic noise
+    r = 256
+    W = torch.randn(r, D, generator=g, device=dev) * (torch.arange(1, r + 1, device=dev) ** -0.7)[:, None]
+    X = torch.empty(count, N, D, dtype=torch.bfloat16, device=dev)
+    for i in range(count):
+        X[i] = (torch.randn(N, r, generator=g, device=dev) @ W + 0.05 * torch.randn(N, D, generator=g, device=dev) + 0.3
+                ).to(torch.bfloat16)
+    ctx = ub.Context(ub.make_shape(1, 1, 1, 1, 256, 128, 8, "bf16"))
+    scratch = torch.empty(ub.lib.uncomp_entropy_wide_scratch_bytes(N, D), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        ub.uncomp_entropy_wide(ctx, X, k, scratch=scratch)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    ub.uncomp_profile_enable(ctx, True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        ent, er = ub.uncomp_entropy_wide(ctx, X, k, scratch=scratch)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    prof = ub.uncomp_profile_read(ctx)
+    ub.uncomp_profile_enable(ctx, False)
+    ms_step = ev0.elapsed_time(ev1) / args.steps
+    nblk = (D + 255) // 256
+    flops_gram = 2.0 * N * 256 * 256 * (nblk * (nblk + 1) // 2)        # block pairs actually computed
+    kernels = {}
+    total_ms = sum(v[0] for v in prof.values())
+    for name, (ms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        avg = ms / cnt
+        ent_k = {"launches_per_step": cnt // args.steps, "avg_ms": round(avg, 4), "share": round(ms / total_ms, 4)}
+        if name == "wide_gram":
+            ach = flops_gram / 1e12 / (avg / 1e3)
+            ent_k.update({"bound": "tensor", "achieved": round(ach, 1), "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                          "frac": round(ach / peaks["bf16_sustained"], 4)})
+        elif name == "wide_tridiag":
+            # the trailing matrix is read and written once per column: (2/3) D^3 floats each way
+            gb = 2.0 * (D ** 3) / 3.0 * 4 / 1e9
+            ent_k.update({"bound": "l2", "achieved": round(gb / (avg / 1e3), 1), "peak": None, "unit": "GB/s of L2 traffic",
+                          "frac": None})
+        else:
+            ent_k["bound"] = "alu"
+        kernels[name] = ent_k
+    launches = sum(c for _, c in prof.values())
+    dom = max(kernels, key=lambda n: kernels[n]["share"])
+    kd = kernels[dom]
+    roofline = {"kernel": dom, "bound": kd["bound"], "achieved": kd.get("achieved"), "peak": kd.get("peak"),
+                "unit": kd.get("unit"), "frac": kd.get("frac"), "traffic": None, "avg_ms": kd["avg_ms"], "share": kd["share"],
+                "peak_source": f"of {peaks['source']} (sustained bf16)"}
+    e2e = None
+    if args.e2e_steps > 0:
+        hX = torch.empty(X.shape, dtype=X.dtype, pin_memory=True).copy_(X)
+        dX = torch.empty_like(X)
+        hout = torch.empty(count, dtype=torch.float32, pin_memory=True)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            dX.copy_(hX, non_blocking=True)
+            en, _ = ub.uncomp_entropy_wide(ctx, dX, k, scratch=scratch)
+            hout.copy_(en, non_blocking=True)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        e2e = {"value": count * N / (e0.elapsed_time(e1) / args.e2e_steps / 1e3), "unit": UNIT,
+               "h2d_bytes_per_step": hX.numel() * 2, "d2h_bytes_per_step": count * 4, "steps": args.e2e_steps}
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        import oracle
+        x0 = X[0].double().cpu().numpy()
+        t0 = time.perf_counter()
+        H, _ = oracle.entropy_wide(x0, k)
+        t_cpu = time.perf_counter() - t0
+        cpu_baseline = {"value": N / t_cpu, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                        "sample": f"1 of {count} matrices (library matmul and eigensolver threads), {t_cpu:.1f} s wall; "
+                                  f"H = {H:.6f}, GPU {float(ent[0]):.6f}"}
+    line = {"metric": "wide_entropy_tokens_per_s", "value": count * N / (ms_step / 1e3), "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"truncated entropy (k {k}) of {count} hidden-state matrices N{N} x D{D} bf16",
+                       "l2": f"inputs {X.numel() * 2 / 1e9:.2f} GB, larger than L2"},
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches,
+            "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
 # ---------------------------------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -629,12 +737,14 @@ def main():
     ap.add_argument("--scale-L", type=int, default=0, help="profiling aid: same recipe with fewer layers")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--path", default="kv", choices=["kv", "hidden", "decode", "prepare"],
+    ap.add_argument("--path", default="kv", choices=["kv", "hidden", "decode", "prepare", "wide"],
                     help="kv: the KV-cache compression pass (the default and the headline); hidden: the "
                          "hidden-state eviction of one layer-group boundary; decode: one decode-time update of "
                          "the compressed cache of every layer; each reported on a line of its own")
     ap.add_argument("--hidden-width", type=int, default=4096)
     ap.add_argument("--hidden-batch", type=int, default=4)
+    ap.add_argument("--wide-N", type=int, default=8192)
+    ap.add_argument("--wide-count", type=int, default=4)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -649,6 +759,9 @@ def main():
         return
     if args.path == "prepare":
         run_prepare(args)
+        return
+    if args.path == "wide":
+        run_wide(args)
         return
 
     import torch

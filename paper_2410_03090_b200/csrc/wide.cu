@@ -12,8 +12,8 @@
 //                        spread over all warps, ONE grid barrier per column.  The rank-2 update of column k
 //                        is applied while the matrix is swept for the matrix-vector product of column k + 1,
 //                        so the matrix (64 MB at D = 4096, resident in L2) is read and written once per column;
-//   5. eigenvalues       Sturm-count multi-section (fp64) for the k largest of the tridiagonal matrix, then
-//                        H_k and erank_k.
+//   5. eigenvalues       Sturm-count 256-section (fp64), one CTA per wanted eigenvalue of the tridiagonal
+//                        matrix, then H_k and erank_k.
 // Every wait is bounded: the TMA / MMA barriers as in the other tensor-core kernels, the grid barrier by a
 // poll limit after which the kernel raises UNCOMP_STATUS_TIMEOUT and all CTAs leave.
 #include <math.h>
@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(256) wide_assemble_kernel(const float *__restr
 }
 
 // ------------------------------------------------------------------------------------- 4. tridiagonalisation
-constexpr int kTriThreads = 512;
+constexpr int kTriThreads = 1024;
 constexpr int kTriWarps = kTriThreads / 32;
 constexpr unsigned kBarrierSpin = 1u << 22;
 
@@ -285,18 +285,29 @@ __global__ void __launch_bounds__(kTriThreads, 1) tridiag_wide_kernel(float *__r
         }
         __syncthreads();                                       // every thread has read vn[k], vn[k + 1]
         for (int j = k + 1 + tid; j < D; j += kTriThreads) vn[j] = (vn[j] - (j == k + 1 ? alpha : 0.f)) * inv;
+        // the sweep below starts at a multiple of four columns: up to three dead columns left of k + 1 ride
+        // along (nobody reads them again) and must not enter the dot product
+        if (tid < 3 && k - tid >= 0) vn[k - tid] = 0.f;
         if (blockIdx.x == 0 && tid == 0) { a_out[k] = (double)akk; e_out[k] = (double)alpha; }
         __syncthreads();
-        // sweep: apply the pending update to rows >= k + 1 and form p = A' vn on the fly
+        // sweep: apply the pending update to rows >= k + 1 and form p = A' vn on the fly, 16 bytes per lane
         float *pw = pbuf + (size_t)(k & 1) * D;
+        const int j0 = (k + 1) & ~3;
         for (int i = k + 1 + gw; i < D; i += total_warps) {
-            const float vi = v[i], wi = w[i];
+            const float vi = -2.f * v[i], wi = -2.f * w[i];
             float *row = A + (size_t)i * D;
             float acc = 0.f;
-            for (int j = k + 1 + lane; j < D; j += 32) {
-                const float x = __ldcg(row + j) - 2.f * (vi * w[j] + wi * v[j]);
-                __stcg(row + j, x);
-                acc = fmaf(x, vn[j], acc);
+#pragma unroll 2
+            for (int j = j0 + 4 * lane; j < D; j += 128) {
+                float4 x = __ldcg(reinterpret_cast<const float4 *>(row + j));
+                const float4 v4 = *reinterpret_cast<const float4 *>(v + j), w4 = *reinterpret_cast<const float4 *>(w + j);
+                const float4 n4 = *reinterpret_cast<const float4 *>(vn + j);
+                x.x = fmaf(vi, w4.x, fmaf(wi, v4.x, x.x));
+                x.y = fmaf(vi, w4.y, fmaf(wi, v4.y, x.y));
+                x.z = fmaf(vi, w4.z, fmaf(wi, v4.z, x.z));
+                x.w = fmaf(vi, w4.w, fmaf(wi, v4.w, x.w));
+                __stcg(reinterpret_cast<float4 *>(row + j), x);
+                acc = fmaf(x.x, n4.x, fmaf(x.y, n4.y, fmaf(x.z, n4.z, fmaf(x.w, n4.w, acc))));
             }
             acc = warp_sum(acc);
             if (lane == 0) __stcg(pw + i, acc);
@@ -342,18 +353,16 @@ __device__ int sturm_count_wide(const double *__restrict__ a, const double *__re
     return cnt;
 }
 
+// grid (k): CTA t finds the t-th largest eigenvalue by 256-section (every CTA repeats the cheap set-up);
+// lam_out[t] and, from CTA 0, the trace in lam_out[k]
 __global__ void __launch_bounds__(kSturmThreads) sturm_wide_kernel(const double *__restrict__ a, const double *__restrict__ e,
-                                                                  int D, int k, int norm, int max_iters,
-                                                                  float *__restrict__ H_out, float *__restrict__ erank_out,
-                                                                  double *__restrict__ spectrum,
+                                                                  int D, int k, int max_iters, double *__restrict__ lam_out,
                                                                   uint32_t *__restrict__ status) {
     __shared__ double redlo[kSturmThreads / 32], redhi[kSturmThreads / 32], redtr[kSturmThreads / 32];
-    __shared__ double xs[kSturmThreads];
-    __shared__ int cs[kSturmThreads];
-    __shared__ double lam[kSturmMaxK];
+    __shared__ int redc[kSturmThreads / 32];
     __shared__ double bounds[3];
-    __shared__ int not_conv;
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    __shared__ int nb_s;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, t = blockIdx.x;
     // Gershgorin interval and trace
     double lo = 1e300, hi = -1e300, tr = 0.0;
     for (int i = tid; i < D; i += kSturmThreads) {
@@ -369,80 +378,75 @@ __global__ void __launch_bounds__(kSturmThreads) sturm_wide_kernel(const double 
         tr += __shfl_xor_sync(0xffffffffu, tr, o);
     }
     if (lane == 0) { redlo[wid] = lo; redhi[wid] = hi; redtr[wid] = tr; }
-    if (tid == 0) not_conv = 0;
     __syncthreads();
     if (tid == 0) {
-        double l = redlo[0], h = redhi[0], t = 0.0;
-        for (int i = 0; i < kSturmThreads / 32; ++i) { l = fmin(l, redlo[i]); h = fmax(h, redhi[i]); t += redtr[i]; }
+        double l = redlo[0], h = redhi[0], sum = 0.0;
+        for (int i = 0; i < kSturmThreads / 32; ++i) { l = fmin(l, redlo[i]); h = fmax(h, redhi[i]); sum += redtr[i]; }
         const double span = fmax(h - l, 1e-300);
         bounds[0] = l - 1e-9 * span;
         bounds[1] = h + 1e-9 * span;
-        bounds[2] = t;
+        bounds[2] = sum;
     }
     __syncthreads();
-    lo = bounds[0];
-    hi = bounds[1];
-    const double radius = fmax(fabs(lo), fabs(hi));
+    double xl = bounds[0], xh = bounds[1];
+    const double radius = fmax(fabs(xl), fabs(xh));
     const double tiny = fmax(radius, 1e-280) * 1e-19;      // floor of a pivot of the Sturm recurrence
     const double tol = radius * 1e-13;
-    // coarse round: 256 points over the interval
-    xs[tid] = lo + (hi - lo) * (double)tid / (double)(kSturmThreads - 1);
-    cs[tid] = sturm_count_wide(a, e, D, xs[tid], tiny);
-    __syncthreads();
-    // teams of 8 lanes refine one eigenvalue each; target t (0 = largest) is ascending index D - 1 - t
-    const int team = tid >> 3, tl = tid & 7, teams = kSturmThreads / 8;
-    const int rounds = max_iters > 0 ? max_iters : 16;
-    for (int t = team; t < k; t += teams) {
-        const int m = D - 1 - t;
-        // bracket from the coarse round: count(xl) <= m < count(xh)
-        int p = 0;
-        for (int s = 0; s < kSturmThreads; ++s)
-            if (cs[s] <= m) p = s;
-        double xl = xs[p], xh = p + 1 < kSturmThreads ? xs[p + 1] : hi;
-        int it = 0;
-        for (; it < rounds && (xh - xl) > tol; ++it) {
-            const double x = xl + (xh - xl) * (double)(tl + 1) / 9.0;
-            const int c = sturm_count_wide(a, e, D, x, tiny);
-            // lanes whose point still has count <= m form a prefix of the team
-            const unsigned shift = (unsigned)(lane & ~7);
-            const unsigned below = (__ballot_sync(0xffu << shift, c <= m) >> shift) & 0xffu;
-            const int nb = __popc(below);
-            const double step = (xh - xl) / 9.0;
-            const double nl = xl + step * (double)nb, nh = nb < 8 ? xl + step * (double)(nb + 1) : xh;
-            xl = nl;
-            xh = nh;
+    const int m = D - 1 - t;                               // ascending index of the wanted eigenvalue
+    // invariant: count(xl) <= m < count(xh).  Each round cuts the bracket into 257 parts.
+    const int rounds = max_iters > 0 ? max_iters : 8;
+    int it = 0;
+    for (; it < rounds && (xh - xl) > tol; ++it) {
+        const double step = (xh - xl) / (double)(kSturmThreads + 1);
+        const int c = sturm_count_wide(a, e, D, xl + step * (double)(tid + 1), tiny);
+        // the points whose count is still <= m form a prefix
+        int below = __popc(__ballot_sync(0xffffffffu, c <= m));
+        if (lane == 0) redc[wid] = below;
+        __syncthreads();
+        if (tid == 0) {
+            int nb = 0;
+            for (int i = 0; i < kSturmThreads / 32; ++i) nb += redc[i];
+            nb_s = nb;
         }
-        if (tl == 0) {
-            lam[t] = 0.5 * (xl + xh);
-            if ((xh - xl) > tol) not_conv = 1;
-        }
+        __syncthreads();
+        const int nb = nb_s;
+        const double nl = xl + step * (double)nb, nh = nb < kSturmThreads ? xl + step * (double)(nb + 1) : xh;
+        xl = nl;
+        xh = nh;
     }
-    __syncthreads();
     if (tid == 0) {
-        if (not_conv) atomicOr(status, (uint32_t)UNCOMP_STATUS_NOT_CONVERGED);
-        double denom = 0.0;
-        if (norm == 0) {
-            for (int i = 0; i < k; ++i) denom += fmax(lam[i], 0.0);
-        } else {
-            denom = bounds[2];
-        }
-        double h = 0.0;
-        for (int i = 0; i < k; ++i) {
-            const double pi = denom > 0.0 ? fmax(lam[i], 0.0) / denom : 0.0;
-            if (pi > 0.0) h -= pi * log(pi);
-        }
-        *H_out = (float)h;
-        if (erank_out) *erank_out = (float)exp(h);
-        if (spectrum)
-            for (int i = 0; i < k; ++i) spectrum[i] = lam[i];
+        lam_out[t] = 0.5 * (xl + xh);
+        if ((xh - xl) > tol) atomicOr(status, (uint32_t)UNCOMP_STATUS_NOT_CONVERGED);
+        if (t == 0) lam_out[k] = bounds[2];
     }
+}
+
+// H_k and erank_k from the k largest eigenvalues (descending) and the trace at lam[k]
+__global__ void wide_entropy_kernel(const double *__restrict__ lam, int k, int norm, float *__restrict__ H_out,
+                                    float *__restrict__ erank_out, double *__restrict__ spectrum) {
+    if (threadIdx.x != 0) return;
+    double denom = 0.0;
+    if (norm == 0) {
+        for (int i = 0; i < k; ++i) denom += fmax(lam[i], 0.0);
+    } else {
+        denom = lam[k];
+    }
+    double h = 0.0;
+    for (int i = 0; i < k; ++i) {
+        const double pi = denom > 0.0 ? fmax(lam[i], 0.0) / denom : 0.0;
+        if (pi > 0.0) h -= pi * log(pi);
+    }
+    *H_out = (float)h;
+    if (erank_out) *erank_out = (float)exp(h);
+    if (spectrum)
+        for (int i = 0; i < k; ++i) spectrum[i] = lam[i];
 }
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WideLayout {
     int nblk, pairs, chunk, chunks;
-    size_t off_bar, off_s, off_colpart, off_a, off_e, off_p, off_C, off_part, bytes;
+    size_t off_bar, off_s, off_colpart, off_a, off_e, off_lam, off_p, off_C, off_part, bytes;
 };
 
 WideLayout wide_layout(int N, int D) {
@@ -461,6 +465,7 @@ WideLayout wide_layout(int N, int D) {
     w.off_colpart = o;  o = align256(o + (size_t)kColChunks * D * sizeof(double));
     w.off_a = o;        o = align256(o + (size_t)D * sizeof(double));
     w.off_e = o;        o = align256(o + (size_t)D * sizeof(double));
+    w.off_lam = o;      o = align256(o + (size_t)(kSturmMaxK + 1) * sizeof(double));
     w.off_p = o;        o = align256(o + (size_t)2 * D * sizeof(float));
     w.off_C = o;        o = align256(o + (size_t)D * D * sizeof(float));
     w.off_part = o;     o = align256(o + (size_t)w.chunks * w.pairs * 2 * 128 * kWBlock * sizeof(float));
@@ -524,8 +529,9 @@ cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const
     {
         ProfScope ps(prof, kSlotWideSturm, st);
         const int k = ep.k_trunc < D ? ep.k_trunc : D;
-        sturm_wide_kernel<<<1, kSturmThreads, 0, st>>>(a, e, D, k, ep.norm, ep.max_iters, d_entropy, d_erank, d_spectrum,
-                                                       d_status);
+        double *lam = (double *)(scratch + w.off_lam);
+        sturm_wide_kernel<<<k, kSturmThreads, 0, st>>>(a, e, D, k, ep.max_iters, lam, d_status);
+        wide_entropy_kernel<<<1, 32, 0, st>>>(lam, k, ep.norm, d_entropy, d_erank, d_spectrum);
     }
     return cudaGetLastError();
 }
