@@ -220,15 +220,22 @@ constexpr int kTriThreads = 1024;
 constexpr int kTriWarps = kTriThreads / 32;
 constexpr unsigned kBarrierSpin = 1u << 22;
 
-__device__ __forceinline__ float tri_block_sum(float v, float *red) {
-    v = warp_sum(v);
-    __syncthreads();                 // red is free again
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+// Three block-wide sums at once, every thread gets the totals (summed in the same order by all).  `red` must not be
+// the array of the previous call: the calls alternate between two arrays, so one barrier per call is enough.
+__device__ __forceinline__ void tri_block_sum3(float &x, float &y, float &z, float (*red)[kTriWarps]) {
+    x = warp_sum(x);
+    y = warp_sum(y);
+    z = warp_sum(z);
+    if ((threadIdx.x & 31) == 0) {
+        red[0][threadIdx.x >> 5] = x;
+        red[1][threadIdx.x >> 5] = y;
+        red[2][threadIdx.x >> 5] = z;
+    }
     __syncthreads();
-    float t = 0.f;
+    float tx = 0.f, ty = 0.f, tz = 0.f;
 #pragma unroll
-    for (int i = 0; i < kTriWarps; ++i) t += red[i];
-    return t;
+    for (int i = 0; i < kTriWarps; ++i) { tx += red[0][i]; ty += red[1][i]; tz += red[2][i]; }
+    x = tx; y = ty; z = tz;
 }
 
 // All CTAs of a cooperative launch meet here.  `bar` counts arrivals monotonically.
@@ -254,43 +261,77 @@ __device__ __forceinline__ bool tri_grid_barrier(unsigned *bar, unsigned &phase,
 
 // A: full symmetric fp32 matrix [D, D], destroyed.  Output: diagonal a[D] and off-diagonal e[D - 1].
 // State at the top of iteration k: rows >= k of A hold the matrix after the reflections of columns 0 .. k - 2;
-// the rank-2 update of column k - 1, A -= 2 (v w^T + w v^T) on rows and columns >= k, is still pending and kept
-// as (v, w) in shared memory by every CTA.
+// the rank-2 update of column k - 1, A -= 2 (v w^T + w v^T) on rows and columns >= k, is still pending: its
+// vector v is in shared memory (vn), the product p = A v it needs is in global memory (written by the last sweep).
+// Every CTA repeats the O(D) vector work of a column (a thread owns up to four columns in registers), so one
+// column costs one grid barrier, two block-wide sums and one sweep over the trailing matrix.
+constexpr int kTriQ = 4;   // columns per thread: D <= kTriQ * kTriThreads
+
 __global__ void __launch_bounds__(kTriThreads, 1) tridiag_wide_kernel(float *__restrict__ A, int D, double *__restrict__ a_out,
                                                                      double *__restrict__ e_out, float *__restrict__ pbuf,
                                                                      unsigned *bar, uint32_t *__restrict__ status) {
     extern __shared__ float sm[];
     float *v = sm, *w = sm + D, *vn = sm + 2 * D;
-    __shared__ float red[kTriWarps];
+    __shared__ float redA[3][kTriWarps], redB[3][kTriWarps];
     __shared__ int flag;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int total_warps = gridDim.x * kTriWarps, gw = blockIdx.x * kTriWarps + warp;
-    for (int i = tid; i < D; i += kTriThreads) { v[i] = 0.f; w[i] = 0.f; }
+    for (int i = tid; i < D; i += kTriThreads) { v[i] = 0.f; w[i] = 0.f; vn[i] = 0.f; }
     __syncthreads();
     unsigned phase = 0;
     for (int k = 0; k + 2 < D; ++k) {
-        // row k with the pending update applied: diagonal entry and the column to eliminate
-        const float vk = v[k], wk = w[k];
-        for (int j = k + tid; j < D; j += kTriThreads)
-            vn[j] = __ldcg(A + (size_t)k * D + j) - 2.f * (vk * w[j] + wk * v[j]);
-        __syncthreads();
-        float part = 0.f;
-        for (int j = k + 1 + tid; j < D; j += kTriThreads) part += vn[j] * vn[j];
-        const float sigma = tri_block_sum(part, red);
-        const float akk = vn[k], x0 = vn[k + 1];
+        // ---- vector work: finish the pending update (w = p - (v . p) v), apply it to row k, next reflection ----
+        const float *pprev = pbuf + (size_t)((k + 1) & 1) * D;
+        float pj[kTriQ], rj[kTriQ];
+#pragma unroll
+        for (int q = 0; q < kTriQ; ++q) {
+            const int j = tid + q * kTriThreads;
+            const bool own = j < D && j >= k;
+            pj[q] = (own && k > 0) ? __ldcg(pprev + j) : 0.f;
+            rj[q] = own ? __ldcg(A + (size_t)k * D + j) : 0.f;
+        }
+        float Kdot = 0.f, pk = 0.f, unused = 0.f;
+#pragma unroll
+        for (int q = 0; q < kTriQ; ++q) {
+            const int j = tid + q * kTriThreads;
+            if (j < D && j >= k) {
+                Kdot = fmaf(vn[j], pj[q], Kdot);
+                if (j == k) pk = pj[q];
+            }
+        }
+        tri_block_sum3(Kdot, pk, unused, redA);
+        const float vk = vn[k], wk = pk - Kdot * vk;
+        float sigma = 0.f, akk = 0.f, x0 = 0.f;
+#pragma unroll
+        for (int q = 0; q < kTriQ; ++q) {
+            const int j = tid + q * kTriThreads;
+            if (j < D && j >= k) {
+                const float vj = vn[j], wj = pj[q] - Kdot * vj;
+                v[j] = vj;
+                w[j] = wj;
+                const float r = rj[q] - 2.f * (vk * wj + wk * vj);
+                rj[q] = r;
+                if (j > k) sigma = fmaf(r, r, sigma);
+                if (j == k) akk = r;
+                if (j == k + 1) x0 = r;
+            }
+        }
+        tri_block_sum3(sigma, akk, x0, redB);     // every thread has read vn[k] before this barrier
         float alpha = 0.f, inv = 0.f;
         if (sigma > 0.f) {
             alpha = -copysignf(sqrtf(sigma), x0);
             inv = 1.f / sqrtf(2.f * (sigma - alpha * x0));     // 1 / |x - alpha e_1|
         }
-        __syncthreads();                                       // every thread has read vn[k], vn[k + 1]
-        for (int j = k + 1 + tid; j < D; j += kTriThreads) vn[j] = (vn[j] - (j == k + 1 ? alpha : 0.f)) * inv;
-        // the sweep below starts at a multiple of four columns: up to three dead columns left of k + 1 ride
-        // along (nobody reads them again) and must not enter the dot product
-        if (tid < 3 && k - tid >= 0) vn[k - tid] = 0.f;
+        // the sweep starts at a multiple of four columns: up to three dead columns left of k + 1 ride along
+        // (nobody reads them again) and must not enter the dot product, hence the zeros
+#pragma unroll
+        for (int q = 0; q < kTriQ; ++q) {
+            const int j = tid + q * kTriThreads;
+            if (j < D && j + 3 >= k) vn[j] = j > k ? (rj[q] - (j == k + 1 ? alpha : 0.f)) * inv : 0.f;
+        }
         if (blockIdx.x == 0 && tid == 0) { a_out[k] = (double)akk; e_out[k] = (double)alpha; }
         __syncthreads();
-        // sweep: apply the pending update to rows >= k + 1 and form p = A' vn on the fly, 16 bytes per lane
+        // ---- sweep: apply the pending update to rows >= k + 1 and form p = A' vn on the fly, 16 bytes per lane ----
         float *pw = pbuf + (size_t)(k & 1) * D;
         const int j0 = (k + 1) & ~3;
         for (int i = k + 1 + gw; i < D; i += total_warps) {
@@ -313,25 +354,17 @@ __global__ void __launch_bounds__(kTriThreads, 1) tridiag_wide_kernel(float *__r
             if (lane == 0) __stcg(pw + i, acc);
         }
         if (!tri_grid_barrier(bar, phase, status, &flag)) return;
-        // new pending update: w = p - (vn . p) vn, v = vn
-        part = 0.f;
-        for (int j = k + 1 + tid; j < D; j += kTriThreads) {
-            const float pj = __ldcg(pw + j);
-            w[j] = pj;
-            part += vn[j] * pj;
-        }
-        const float Kdot = tri_block_sum(part, red);
-        for (int j = k + 1 + tid; j < D; j += kTriThreads) {
-            w[j] -= Kdot * vn[j];
-            v[j] = vn[j];
-        }
-        __syncthreads();
     }
+    // the last 2 x 2 block: its pending update comes from column D - 3
     if (blockIdx.x == 0 && tid == 0) {
         const int i = D - 2, j = D - 1;
-        a_out[i] = (double)(__ldcg(A + (size_t)i * D + i) - 4.f * v[i] * w[i]);
-        e_out[i] = (double)(__ldcg(A + (size_t)i * D + j) - 2.f * (v[i] * w[j] + w[i] * v[j]));
-        a_out[j] = (double)(__ldcg(A + (size_t)j * D + j) - 4.f * v[j] * w[j]);
+        const float *pprev = pbuf + (size_t)((D - 3) & 1) * D;
+        const float pi = __ldcg(pprev + i), pjv = __ldcg(pprev + j);
+        const float Kdot = vn[i] * pi + vn[j] * pjv;
+        const float wi = pi - Kdot * vn[i], wj = pjv - Kdot * vn[j];
+        a_out[i] = (double)(__ldcg(A + (size_t)i * D + i) - 4.f * vn[i] * wi);
+        e_out[i] = (double)(__ldcg(A + (size_t)i * D + j) - 2.f * (vn[i] * wj + wi * vn[j]));
+        a_out[j] = (double)(__ldcg(A + (size_t)j * D + j) - 4.f * vn[j] * wj);
     }
 }
 

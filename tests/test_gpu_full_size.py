@@ -69,3 +69,30 @@ def test_full_size_workload(name, n_float, n_select):
             assert b[l, l % 8] == b[l].max()
     del K, V, Qw, cp, out
     torch.cuda.empty_cache()
+
+
+def test_full_size_wide_entropy_hidden_states():
+    """Hidden-state shape of the 8B models (D = 4096) at 8192 tokens, the size `bench.py --path wide` times: the
+    entropy and the 32 largest eigenvalues against the oracle, plus properties that hold at any size."""
+    import oracle
+    from paper_2410_03090_b200 import binding as ub
+    N, D, k = 8192, 4096, 32
+    g = torch.Generator(device="cuda").manual_seed(11)
+    W = torch.randn(256, D, generator=g, device="cuda") * (torch.arange(1, 257, device="cuda") ** -0.7)[:, None]
+    X = (torch.randn(N, 256, generator=g, device="cuda") @ W + 0.05 * torch.randn(N, D, generator=g, device="cuda") + 0.3
+         ).to(torch.bfloat16)[None]
+    ctx = ub.Context(ub.make_shape(1, 1, 1, 1, 256, 128, 8, "bf16"))
+    ent, er, spec = ub.uncomp_entropy_wide(ctx, X, k, spectrum=True)
+    ent1, _, spec1 = ub.uncomp_entropy_wide(ctx, X, k, norm=1, spectrum=True)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    H, E, lam = oracle.entropy_wide(X[0].double().cpu().numpy(), k, return_spectrum=True)
+    got = spec[0].cpu().numpy()
+    assert np.abs(got - lam[:k]).max() <= 1e-4 * lam[0]
+    assert abs(float(ent[0]) - H) <= parity.ENTROPY_RTOL * max(abs(H), 1.0)
+    assert abs(float(er[0]) - E) <= 2e-4 * E
+    # descending, non-negative, H_k <= ln k, same bits on a second run, whole-trace normalisation gives less entropy mass
+    assert (np.diff(got) <= 0).all() and got[-1] > 0 and 0.0 <= float(ent[0]) <= np.log(k) + 1e-6
+    assert torch.equal(spec, spec1) and float(ent1[0]) != float(ent[0])
+    H1 = oracle.truncated_entropy(lam, k, 1)[0]
+    assert abs(float(ent1[0]) - H1) <= parity.ENTROPY_RTOL * max(abs(H1), 1.0)
