@@ -220,22 +220,24 @@ constexpr int kTriThreads = 1024;
 constexpr int kTriWarps = kTriThreads / 32;
 constexpr unsigned kBarrierSpin = 1u << 22;
 
-// Three block-wide sums at once, every thread gets the totals (summed in the same order by all).  `red` must not be
-// the array of the previous call: the calls alternate between two arrays, so one barrier per call is enough.
-__device__ __forceinline__ void tri_block_sum3(float &x, float &y, float &z, float (*red)[kTriWarps]) {
+// Three block-wide sums at once; every thread gets the totals.  Warp 0 adds the per-warp sums (a butterfly: a fixed
+// order) and publishes them.  `red` must not be the array of the previous call: the calls alternate between two
+// arrays, which saves the barrier that would otherwise protect the array's reuse.
+__device__ __forceinline__ void tri_block_sum3(float &x, float &y, float &z, float (*red)[kTriWarps + 1]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     x = warp_sum(x);
     y = warp_sum(y);
     z = warp_sum(z);
-    if ((threadIdx.x & 31) == 0) {
-        red[0][threadIdx.x >> 5] = x;
-        red[1][threadIdx.x >> 5] = y;
-        red[2][threadIdx.x >> 5] = z;
+    if (lane == 0) { red[0][warp] = x; red[1][warp] = y; red[2][warp] = z; }
+    __syncthreads();
+    if (warp == 0) {
+        float tx = warp_sum(red[0][lane]), ty = warp_sum(red[1][lane]), tz = warp_sum(red[2][lane]);
+        if (lane == 0) { red[0][kTriWarps] = tx; red[1][kTriWarps] = ty; red[2][kTriWarps] = tz; }
     }
     __syncthreads();
-    float tx = 0.f, ty = 0.f, tz = 0.f;
-#pragma unroll
-    for (int i = 0; i < kTriWarps; ++i) { tx += red[0][i]; ty += red[1][i]; tz += red[2][i]; }
-    x = tx; y = ty; z = tz;
+    x = red[0][kTriWarps];
+    y = red[1][kTriWarps];
+    z = red[2][kTriWarps];
 }
 
 // All CTAs of a cooperative launch meet here.  `bar` counts arrivals monotonically.
@@ -272,7 +274,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) tridiag_wide_kernel(float *__r
                                                                      unsigned *bar, uint32_t *__restrict__ status) {
     extern __shared__ float sm[];
     float *v = sm, *w = sm + D, *vn = sm + 2 * D;
-    __shared__ float redA[3][kTriWarps], redB[3][kTriWarps];
+    __shared__ float redA[3][kTriWarps + 1], redB[3][kTriWarps + 1];
     __shared__ int flag;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int total_warps = gridDim.x * kTriWarps, gw = blockIdx.x * kTriWarps + warp;
@@ -338,17 +340,27 @@ __global__ void __launch_bounds__(kTriThreads, 1) tridiag_wide_kernel(float *__r
             const float vi = -2.f * v[i], wi = -2.f * w[i];
             float *row = A + (size_t)i * D;
             float acc = 0.f;
-#pragma unroll 2
-            for (int j = j0 + 4 * lane; j < D; j += 128) {
-                float4 x = __ldcg(reinterpret_cast<const float4 *>(row + j));
-                const float4 v4 = *reinterpret_cast<const float4 *>(v + j), w4 = *reinterpret_cast<const float4 *>(w + j);
-                const float4 n4 = *reinterpret_cast<const float4 *>(vn + j);
-                x.x = fmaf(vi, w4.x, fmaf(wi, v4.x, x.x));
-                x.y = fmaf(vi, w4.y, fmaf(wi, v4.y, x.y));
-                x.z = fmaf(vi, w4.z, fmaf(wi, v4.z, x.z));
-                x.w = fmaf(vi, w4.w, fmaf(wi, v4.w, x.w));
-                __stcg(reinterpret_cast<float4 *>(row + j), x);
-                acc = fmaf(x.x, n4.x, fmaf(x.y, n4.y, fmaf(x.z, n4.z, fmaf(x.w, n4.w, acc))));
+            for (int jb = j0 + 4 * lane; jb < D; jb += 512) {      // batches of four loads in flight per lane
+                float4 x[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    x[u] = jb + u * 128 < D ? __ldcg(reinterpret_cast<const float4 *>(row + jb + u * 128))
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int j = jb + u * 128;
+                    if (j < D) {
+                        const float4 v4 = *reinterpret_cast<const float4 *>(v + j), w4 = *reinterpret_cast<const float4 *>(w + j);
+                        const float4 n4 = *reinterpret_cast<const float4 *>(vn + j);
+                        float4 y = x[u];
+                        y.x = fmaf(vi, w4.x, fmaf(wi, v4.x, y.x));
+                        y.y = fmaf(vi, w4.y, fmaf(wi, v4.y, y.y));
+                        y.z = fmaf(vi, w4.z, fmaf(wi, v4.z, y.z));
+                        y.w = fmaf(vi, w4.w, fmaf(wi, v4.w, y.w));
+                        __stcg(reinterpret_cast<float4 *>(row + j), y);
+                        acc = fmaf(y.x, n4.x, fmaf(y.y, n4.y, fmaf(y.z, n4.z, fmaf(y.w, n4.w, acc))));
+                    }
+                }
             }
             acc = warp_sum(acc);
             if (lane == 0) __stcg(pw + i, acc);
