@@ -277,7 +277,8 @@ __global__ void __launch_bounds__(kTriThreads, 1) tridiag_wide_kernel(float *__r
     __shared__ float redA[3][kTriWarps + 1], redB[3][kTriWarps + 1];
     __shared__ int flag;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int total_warps = gridDim.x * kTriWarps, gw = blockIdx.x * kTriWarps + warp;
+    // rows go round-robin over the CTAs first, so that a short trailing matrix still keeps every SM busy
+    const int total_warps = gridDim.x * kTriWarps, gw = warp * gridDim.x + blockIdx.x;
     for (int i = tid; i < D; i += kTriThreads) { v[i] = 0.f; w[i] = 0.f; vn[i] = 0.f; }
     __syncthreads();
     unsigned phase = 0;
