@@ -24,17 +24,43 @@ namespace uncomp {
 
 namespace {
 // ------------------------------------------------------------------------------------------ 1. column sums
-constexpr int kColChunks = 32;
+constexpr int kColChunks = 64;
 
+// grid (D / 128 feature groups, token chunks), 8 warps: a lane owns 4 adjacent features (one 8-byte load per token
+// row, a warp reads 256 contiguous bytes), warp w takes the tokens t0 + w, t0 + w + 8, ...; the 8 warps are added
+// in warp order
 __global__ void __launch_bounds__(256) wide_colsum_kernel(const __nv_bfloat16 *__restrict__ X, int64_t sN, int N, int D,
                                                          double *__restrict__ part) {
-    const int f = blockIdx.x * 256 + threadIdx.x, c = blockIdx.y;
-    if (f >= D) return;
+    __shared__ double red[8][128];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int f = blockIdx.x * 128 + lane * 4, c = blockIdx.y;
     const int per = (N + kColChunks - 1) / kColChunks;
     const int t0 = c * per, t1 = min(N, t0 + per);
-    double acc = 0.0;
-    for (int t = t0; t < t1; ++t) acc += (double)__bfloat162float(X[(int64_t)t * sN + f]);
-    part[(size_t)c * D + f] = acc;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    if (f < D) {
+        for (int t = t0 + warp; t < t1; t += 32) {
+            uint2 x[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                x[u] = t + 8 * u < t1 ? *reinterpret_cast<const uint2 *>(X + (int64_t)(t + 8 * u) * sN + f) : make_uint2(0u, 0u);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                acc[0] += (double)__uint_as_float(x[u].x << 16);
+                acc[1] += (double)__uint_as_float(x[u].x & 0xffff0000u);
+                acc[2] += (double)__uint_as_float(x[u].y << 16);
+                acc[3] += (double)__uint_as_float(x[u].y & 0xffff0000u);
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) red[warp][lane * 4 + i] = acc[i];
+    __syncthreads();
+    if (threadIdx.x < 128 && blockIdx.x * 128 + threadIdx.x < D) {
+        double sum = 0.0;
+#pragma unroll
+        for (int wv = 0; wv < 8; ++wv) sum += red[wv][threadIdx.x];
+        part[(size_t)c * D + blockIdx.x * 128 + threadIdx.x] = sum;
+    }
 }
 
 __global__ void __launch_bounds__(256) wide_colsum_reduce_kernel(const double *__restrict__ part, int D,
@@ -535,7 +561,7 @@ cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const
     if (err != cudaSuccess) return err;
     {
         ProfScope ps(prof, kSlotWideGram, st);
-        wide_colsum_kernel<<<dim3((D + 255) / 256, kColChunks), 256, 0, st>>>(X, sN, N, D, colpart);
+        wide_colsum_kernel<<<dim3((D + 127) / 128, kColChunks), 256, 0, st>>>(X, sN, N, D, colpart);
         wide_colsum_reduce_kernel<<<(D + 255) / 256, 256, 0, st>>>(colpart, D, s);
         CUtensorMap tmap;
         uint64_t dims[3] = {(uint64_t)D, (uint64_t)N, 1};
@@ -565,8 +591,7 @@ cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const
         if (err != cudaSuccess) return err;
         if (per_sm < 1) return cudaErrorLaunchOutOfResources;
         int grid = sms;                                          // one CTA per SM: all of them are resident
-        const int rows_warps = (D + kTriWarps - 1) / kTriWarps;  // no more CTAs than there are rows to share
-        if (grid > rows_warps) grid = rows_warps;
+        if (grid > D / 8) grid = D / 8;                           // small matrices: fewer CTAs, cheaper barrier
         int Di = D;
         void *args[] = {(void *)&C, (void *)&Di, (void *)&a, (void *)&e, (void *)&pbuf, (void *)&bar, (void *)&d_status};
         err = cudaLaunchCooperativeKernel((const void *)tridiag_wide_kernel, dim3(grid), dim3(kTriThreads), args, smem, st);
