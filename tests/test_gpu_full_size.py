@@ -96,3 +96,75 @@ def test_full_size_wide_entropy_hidden_states():
     assert torch.equal(spec, spec1) and float(ent1[0]) != float(ent[0])
     H1 = oracle.truncated_entropy(lam, k, 1)[0]
     assert abs(float(ent1[0]) - H1) <= parity.ENTROPY_RTOL * max(abs(H1), 1.0)
+
+
+def test_full_size_hidden_state_eviction():
+    """The configuration `bench.py --path hidden` times (B4, 32 query / 8 KV heads, N 32768, D 4096, keep half):
+    scores of one sequence against the oracle, selection and gathered rows of every sequence."""
+    import oracle
+    from paper_2410_03090_b200 import binding as ub
+    wl = synth.scaled(synth.WORKLOADS["c3"], L=1, B=4)
+    D, n_keep = 4096, wl.N // 2
+    K, _, Qw = synth.generate(wl, "cuda")
+    Kl, q = K[:, 0], Qw[:, 0, :, -1, :].contiguous()
+    X = synth.hidden_states(wl, D, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, 1, wl.H, wl.Hq, wl.N, wl.d, 1, wl.dtype))
+    scores = torch.empty(wl.B, wl.N - 1, device="cuda")
+    idx, Xout = ub.uncomp_evict_hidden(ctx, q, Kl, X, n_keep, scores=scores)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    ref = oracle.last_token_scores(q[1].double().cpu().numpy(), Kl[1].double().cpu().numpy())
+    got = scores[1].double().cpu().numpy()
+    assert (np.abs(got - ref[:-1]) <= parity.SCORE_RTOL * np.abs(ref[:-1]) + 1e-12 * ref.max()).all()
+    assert abs(ref.sum() - wl.Hq) < 1e-9                         # every head's attention sums to one
+    for b in range(wl.B):
+        want = oracle.select(scores[b].double().cpu().numpy(), 1, n_keep)
+        np.testing.assert_array_equal(idx[b].cpu().numpy(), want)
+        assert torch.equal(Xout[b], X[b][idx[b].long()])
+
+
+def test_full_size_decode_update_after_prefill():
+    """The state `bench.py --path decode` starts from (the compressed cache of workload c3 after its prefill pass):
+    three decode steps, sampled units against the oracle, invariants on all units."""
+    import oracle
+    from paper_2410_03090_b200 import binding as ub
+    from paper_2410_03090_b200.compress import CompressionPass
+    wl = synth.WORKLOADS["c3"]
+    K, V, Qw = synth.generate(wl, "cuda")
+    cp = CompressionPass(wl, "cuda")
+    o = cp.run(K, V, Qw)
+    torch.cuda.synchronize()
+    offs = o.offsets.cpu().numpy()
+    g = torch.Generator(device="cuda").manual_seed(3)
+    cum = torch.rand(wl.total_rows, generator=g, device="cuda")
+    pos, lens = o.indices.clone(), o.budgets.reshape(-1).clone()
+    Kc, Vc = o.Kc.clone(), o.Vc.clone()
+    max_cap = int(lens.max())
+    sample = [0, 7, 100, 255]
+    for step in range(3):
+        qn = Qw[:, :, :, -1 - step, :].contiguous()
+        kn, vn = K[:, :, :, -1 - step, :].contiguous(), V[:, :, :, -1 - step, :].contiguous()
+        before = {u: (Kc[offs[u]:offs[u + 1]].double().cpu().numpy(), pos[offs[u]:offs[u + 1]].cpu().numpy(),
+                      cum[offs[u]:offs[u + 1]].cpu().numpy()) for u in sample}
+        pos_all = pos.clone()
+        p = torch.empty(wl.total_rows + wl.units, device="cuda")
+        ev = torch.empty(wl.units, dtype=torch.int32, device="cuda")
+        npos = torch.full((wl.B,), wl.N + step, dtype=torch.int32, device="cuda")
+        ub.uncomp_decode_update(cp.ctx, qn, kn, vn, npos, o.offsets, lens, max_cap, Kc, Vc, pos, cum, p=p, evicted=ev)
+        torch.cuda.synchronize()
+        assert cp.status() == 0
+        for u in sample:
+            Kb, pb, cb = before[u]
+            n = len(pb)
+            ref = oracle.decode_probs(qn.view(wl.units, wl.G, wl.d)[u].double().cpu().numpy(), Kb,
+                                      kn.view(wl.units, wl.d)[u].double().cpu().numpy())
+            got = p[offs[u] + u:offs[u] + u + n + 1].cpu().numpy()
+            assert (np.abs(got - ref) <= parity.SCORE_RTOL * np.abs(ref) + 1e-12 * ref.max()).all()
+            slot = oracle.decode_evict((cb + got[:n]).astype(np.float64), pb, wl.N + step, 1)
+            assert int(ev[u]) == int(pb[slot]) and int(pos[offs[u] + slot]) == wl.N + step
+            assert torch.equal(Kc[offs[u] + slot], kn.view(wl.units, wl.d)[u])
+        # every unit: full caches stay full, exactly one position per unit changed, the evicted one is gone
+        assert torch.equal(lens, o.budgets.reshape(-1))
+        changed = (pos != pos_all).cpu().numpy()
+        assert changed.sum() == wl.units and (np.add.reduceat(changed, offs[:-1]) == 1).all()
+        assert (pos[torch.from_numpy(changed).cuda()] == wl.N + step).all()
