@@ -27,8 +27,8 @@ if ROOT not in sys.path:
 # DRAM bytes per (unit x token) of one launch, dram__bytes_read.sum + dram__bytes_write.sum from the ncu capture
 # summarised in profiles/kernels_c3_N16384_L10_ncu_full.md (80 units x 16384 tokens; traffic grows with
 # units x tokens, so a full-size launch is scaled by that product).  Set to None when a kernel changes.
-TRAFFIC_PER_UNIT_TOKEN = {"gram_score_stats": (340.92e6 + 33.37e6) / (80 * 16384),
-                          "score_colsum": (341.00e6 + 7.15e6) / (80 * 16384)}
+TRAFFIC_PER_UNIT_TOKEN = {"gram_score_stats": (341.02e6 + 33.73e6) / (80 * 16384),
+                          "score_colsum": (340.94e6 + 7.60e6) / (80 * 16384)}
 EXP_KERNELS = ("score_stats", "score_colsum", "gram_score_stats")
 METRIC = "compression_pass_tokens_per_s"
 UNIT = "tokens/s"
