@@ -45,6 +45,8 @@ _lib.oracle_group_labels.argtypes = [_dp, C.c_int, C.c_int, C.c_int, C.c_int, _i
 _lib.oracle_group_labels.restype = C.c_int
 _lib.oracle_majority_vote.argtypes = [_dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, _i32p, _i32p]
 _lib.oracle_majority_vote.restype = C.c_int
+_lib.oracle_decode_seed.argtypes = [_dp, C.c_int, _i32p, C.c_int, _dp]
+_lib.oracle_decode_seed.restype = None
 _lib.oracle_pool.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _dp]
 _lib.oracle_pool.restype = None
 _lib.oracle_select.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _i32p]
@@ -258,3 +260,13 @@ def entropy_wide(X, k_trunc: int = 32, center: bool = True, norm: int = 0, retur
     if return_spectrum:
         return H, E, lam
     return H, E
+
+
+def decode_seed(score, idx) -> np.ndarray:
+    """Cumulative scores of one head's cache after prefill: score [P] of the prefix positions, idx the kept
+    positions (window positions are >= P) -> cum [len(idx)]."""
+    score = _f64(score)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    cum = np.empty(len(idx), dtype=np.float64)
+    _lib.oracle_decode_seed(_p(score, _dp), len(score), _p(idx, _i32p), len(idx), _p(cum, _dp))
+    return cum

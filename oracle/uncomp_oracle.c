@@ -523,3 +523,22 @@ int oracle_majority_vote(const double *erank, int S, int L, int H, int M, int sc
     free(one);
     return 0;
 }
+
+
+/* ----------------------------------------------------------------------------------------------
+ * Cumulative scores of a head's cache right after prefill (Section 3.3.3, "Dynamic KV Cache Eviction":
+ * the cumulative attention score window is what decides evictions during decoding).
+ * score is the head's prefill score of every prefix position [P]; idx [n] the kept positions (prefix
+ * positions < P and the w window positions >= P).  A kept prefix position starts with its prefill score.
+ * Reading: the paper does not score the window positions themselves (they are kept unconditionally at
+ * prefill); each starts with the largest score among the kept prefix positions of its head (0 if none
+ * is kept), so a window token never leaves before a prefix token merely for lack of a score.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_decode_seed(const double *score, int P, const int32_t *idx, int n, double *cum)
+{
+    double top = 0.0;
+    int any = 0;
+    for (int t = 0; t < n; ++t)
+        if (idx[t] < P && (!any || score[idx[t]] > top)) { top = score[idx[t]]; any = 1; }
+    for (int t = 0; t < n; ++t) cum[t] = idx[t] < P ? score[idx[t]] : top;
+}

@@ -119,3 +119,13 @@ def test_update_appends_below_budget_and_evicts_at_budget():
     assert ev3 == 2 and list(pos3) == [0, 3, 7, 8, 9, 10] and len(cum3) == 6      # entry with cum 0.01 + p < rest
     assert (K3[-1] == kn).all() and (V3[:5] == Vc[[0, 2, 3, 4, 5]]).all()
     np.testing.assert_allclose(cum3[:5], (cum + p3[:6])[[0, 2, 3, 4, 5]], rtol=1e-15)
+
+
+def test_seed_of_the_cumulative_scores():
+    score = np.array([0.5, 0.1, 0.9, 0.3, 0.7])                 # P = 5
+    np.testing.assert_array_equal(oracle.decode_seed(score, [1, 3, 5, 6]), [0.1, 0.3, 0.3, 0.3])
+    np.testing.assert_array_equal(oracle.decode_seed(score, [2, 4, 5]), [0.9, 0.7, 0.9])
+    np.testing.assert_array_equal(oracle.decode_seed(score, [5, 6]), [0.0, 0.0])          # only the window is kept
+    np.testing.assert_array_equal(oracle.decode_seed(-score, [0, 1, 7]), [-0.5, -0.1, -0.1])   # negative scores: still the largest
+    # kept positions need not be sorted
+    np.testing.assert_array_equal(oracle.decode_seed(score, [6, 0, 2]), [0.9, 0.5, 0.9])
