@@ -398,16 +398,9 @@ def run_decode(args):
     o = cp.run(K, V, Qw)
     torch.cuda.synchronize()
     assert cp.status() == 0
-    # state after prefill: full caches; cumulative scores seeded with the prefill scores of the kept prefix
-    # tokens and, for the window tokens (which the prefill does not score), the largest of them
+    # state after prefill: full caches; cumulative scores seeded from the prefill scores
     offs = o.offsets.cpu().numpy()
-    P = wl.N - wl.w
-    cum = torch.empty(wl.total_rows, device=dev)
-    sc = o.scores.view(wl.units, P)
-    for u in range(wl.units):
-        idx = o.indices[offs[u]:offs[u + 1]].long()
-        pre = idx < P
-        cum[offs[u]:offs[u + 1]] = torch.where(pre, sc[u][idx.clamp(max=P - 1)], sc[u].max())
+    cum = ub.uncomp_decode_seed(cp.ctx, o.scores, o.indices, o.offsets)
     pos = o.indices.clone()
     lens = o.budgets.reshape(-1).clone()
     Kc, Vc = o.Kc, o.Vc

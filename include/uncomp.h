@@ -266,6 +266,24 @@ int uncomp_evict_hidden(uncomp_ctx *ctx, const void *d_qlast, const void *d_K, u
                         void *stream);
 
 /* ---------------------------------------------------------------------------------------------------
+ * uncomp_decode_seed -- Section 3.3.3 "Dynamic KV Cache Eviction": the cumulative attention scores that
+ * decide evictions during decoding start from the prefill's window scores.  For every unit, row t of its
+ * slab of the ragged cache (position indices[offsets[u] + t]) gets
+ *   cum = scores[u, position]                               for a kept prefix position (< N - w)
+ *   cum = max over the unit's kept prefix positions of scores[u, .]   for a window position (0 if the unit
+ *         keeps no prefix position)
+ * Reading: the prefill does not score the window positions (they are kept unconditionally); giving them
+ * the head's largest kept score means a window token is never evicted before a prefix token merely for
+ * lack of a score.  d_pos of uncomp_decode_update is d_indices itself (copy it: the update changes it).
+ *
+ * d_scores   in   [B, L, H, N - w] float, the d_scores output of uncomp_score_select
+ * d_indices  in   [offsets[units]] int32;  d_offsets in [B*L*H + 1] int64 (outputs of the same call)
+ * d_cum      out  [offsets[units]] float
+ * ------------------------------------------------------------------------------------------------- */
+int uncomp_decode_seed(uncomp_ctx *ctx, const float *d_scores, const int32_t *d_indices, const int64_t *d_offsets,
+                       float *d_cum, void *stream);
+
+/* ---------------------------------------------------------------------------------------------------
  * uncomp_decode_update -- Section 3.3.3 "Dynamic KV Cache Eviction", last sentence (as new tokens are
  * generated, the token with the lowest cumulative attention score is evicted) and Algorithm 2, decoding
  * loop (the new token is concatenated with each head's cache and attends over the concatenation).

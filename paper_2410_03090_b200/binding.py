@@ -89,6 +89,8 @@ def _load() -> C.CDLL:
                                         C.POINTER(uncomp_entropy_params), vp, C.c_size_t, fp, fp, dp, vp]
     lib.uncomp_prepare_groups.restype = C.c_int
     lib.uncomp_prepare_groups.argtypes = [vp, fp, C.c_int32, C.c_int32, C.c_int32, fp, i32p, i32p, i32p, vp]
+    lib.uncomp_decode_seed.restype = C.c_int
+    lib.uncomp_decode_seed.argtypes = [vp, fp, i32p, i64p, fp, vp]
     lib.uncomp_decode_update.restype = C.c_int
     lib.uncomp_decode_update.argtypes = [vp, vp, vp, vp, i32p, i64p, i32p, C.c_int32, C.c_int64, C.c_int32, C.c_float,
                                          vp, vp, i32p, fp, fp, i32p, vp]
@@ -259,6 +261,16 @@ def uncomp_evict_hidden(ctx: Context, qlast: torch.Tensor, K_layer: torch.Tensor
     _check(lib.uncomp_evict_hidden(ctx.handle, _ptr(qlast), _ptr(K_layer), st, _ptr(X), D, n_keep, scale, _ptr(scores),
                                    _ptr(indices), _ptr(Xout), _stream(stream)), "uncomp_evict_hidden")
     return indices, Xout
+
+
+def uncomp_decode_seed(ctx: Context, scores: torch.Tensor, indices: torch.Tensor, offsets: torch.Tensor,
+                       cum: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Cumulative scores of the ragged cache right after prefill, from the outputs of uncomp_score_select."""
+    if cum is None:
+        cum = torch.empty(indices.shape[0], dtype=torch.float32, device=indices.device)
+    _check(lib.uncomp_decode_seed(ctx.handle, _ptr(scores), _ptr(indices), _ptr(offsets), _ptr(cum), _stream(stream)),
+           "uncomp_decode_seed")
+    return cum
 
 
 def uncomp_decode_update(ctx: Context, qnew: torch.Tensor, knew: torch.Tensor, vnew: torch.Tensor,

@@ -384,6 +384,14 @@ int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_str
     return UNCOMP_OK;
 }
 
+int uncomp_decode_seed(uncomp_ctx *ctx, const float *d_scores, const int32_t *d_indices, const int64_t *d_offsets,
+                       float *d_cum, void *stream) {
+    if (!ctx || !d_scores || !d_indices || !d_offsets || !d_cum) return UNCOMP_E_NULL;
+    cudaError_t e = launch_decode_seed(ctx->plan, d_scores, d_indices, d_offsets, d_cum, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
 int uncomp_decode_update(uncomp_ctx *ctx, const void *d_qnew, const void *d_knew, const void *d_vnew,
                          const int32_t *d_new_pos, const int64_t *d_offsets, int32_t *d_lens, int32_t max_cap,
                          int64_t total_cap, int32_t protect, float scale, void *d_Kc, void *d_Vc, int32_t *d_pos,

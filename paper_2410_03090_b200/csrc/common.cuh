@@ -106,6 +106,8 @@ cudaError_t launch_evict_hidden(const Plan &p, const void *d_qlast, const void *
                                 const void *d_X, int64_t row_bytes, int n_keep, float scale, float *d_logits,
                                 float *d_stats, float *d_raw, int32_t *d_budgets, int64_t *d_offsets, float *d_scores,
                                 int32_t *d_indices, void *d_Xout, uint32_t *d_status, Profiler *prof, cudaStream_t st);
+cudaError_t launch_decode_seed(const Plan &p, const float *d_scores, const int32_t *d_indices, const int64_t *d_offsets,
+                               float *d_cum, cudaStream_t st);
 int decode_chunks(int max_cap);
 size_t decode_partial_bytes();
 cudaError_t launch_decode_update(const Plan &p, const void *d_q, const void *d_knew, const void *d_vnew,

@@ -342,7 +342,41 @@ __global__ void __launch_bounds__(64) decode_commit_kernel(DecArgs a, int H_per_
     if (tid < 32) { if (tid < vecs) dstK[tid] = srcK[tid]; }
     else if (tid - 32 < vecs) dstV[tid - 32] = srcV[tid - 32];
 }
+// Cumulative scores right after prefill: a kept prefix position takes its prefill score, a window position the
+// largest score among the kept prefix positions of its head (0 if there is none).  One CTA per unit.
+__global__ void __launch_bounds__(256) decode_seed_kernel(const float *__restrict__ scores, int P,
+                                                         const int32_t *__restrict__ indices,
+                                                         const int64_t *__restrict__ offsets, float *__restrict__ cum) {
+    __shared__ float red[8];
+    const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int64_t off = offsets[u];
+    const int n = (int)(offsets[u + 1] - off);
+    const float *s = scores + (size_t)u * P;
+    float top = -INFINITY;
+    for (int t = tid; t < n; t += 256) {
+        const int j = indices[off + t];
+        if (j < P) top = fmaxf(top, s[j]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, o));
+    if (lane == 0) red[wid] = top;
+    __syncthreads();
+    top = red[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) top = fmaxf(top, red[i]);
+    if (top == -INFINITY) top = 0.f;
+    for (int t = tid; t < n; t += 256) {
+        const int j = indices[off + t];
+        cum[off + t] = j < P ? s[j] : top;
+    }
+}
 }  // namespace
+
+cudaError_t launch_decode_seed(const Plan &p, const float *d_scores, const int32_t *d_indices, const int64_t *d_offsets,
+                               float *d_cum, cudaStream_t st) {
+    decode_seed_kernel<<<p.units, 256, 0, st>>>(d_scores, p.prefix, d_indices, d_offsets, d_cum);
+    return cudaGetLastError();
+}
 
 int decode_chunks(int max_cap) { return (max_cap + 1 + kDecChunk - 1) / kDecChunk; }
 size_t decode_partial_bytes() { return sizeof(MinPair); }

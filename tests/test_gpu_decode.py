@@ -157,3 +157,28 @@ def test_decode_rejections_and_bad_unit():
     with pytest.raises(ub.UncompError) as ei:
         ub.uncomp_decode_update(big, q2, k2, v2, npos, st2.offsets, st2.lens, 400, st2.Kc, st2.Vc, st2.pos, st2.cum)
     assert ei.value.code == ub.UNCOMP_E_LIMIT
+
+
+def test_decode_seed_matches_oracle():
+    from paper_2410_03090_b200 import binding as ub
+    from paper_2410_03090_b200 import synth
+    from paper_2410_03090_b200.compress import CompressionPass
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=2048, L=2)
+    K, V, Qw = synth.generate(wl, "cuda")
+    cp = CompressionPass(wl, "cuda")
+    o = cp.run(K, V, Qw)
+    cum = ub.uncomp_decode_seed(cp.ctx, o.scores, o.indices, o.offsets)
+    torch.cuda.synchronize()
+    offs = o.offsets.cpu().numpy()
+    sc = o.scores.reshape(wl.units, -1).double().cpu().numpy()
+    idx = o.indices.cpu().numpy()
+    got = cum.cpu().numpy()
+    for u in range(wl.units):
+        want = oracle.decode_seed(sc[u], idx[offs[u]:offs[u + 1]])
+        np.testing.assert_array_equal(got[offs[u]:offs[u + 1]], want.astype(np.float32))
+    # a unit that keeps only its window: every row starts at 0
+    ctx = ub.Context(ub.make_shape(1, 1, 1, 1, 64, 128, 8, "bf16"))
+    scores = torch.rand(1, 1, 1, 56, device="cuda")
+    idx1 = torch.arange(56, 64, dtype=torch.int32, device="cuda")
+    off1 = torch.tensor([0, 8], dtype=torch.int64, device="cuda")
+    assert float(ub.uncomp_decode_seed(ctx, scores, idx1, off1).abs().max()) == 0.0
