@@ -14,6 +14,10 @@
 //                        so the matrix (64 MB at D = 4096, resident in L2) is read and written once per column;
 //   5. eigenvalues       Sturm-count 256-section (fp64), one CTA per wanted eigenvalue of the tridiagonal
 //                        matrix, then H_k and erank_k.
+// When the matrix has fewer tokens than features (N < D) the same non-zero eigenvalues are taken from the N x N
+// matrix of the centred rows' inner products, (x_i - mean) . (x_j - mean) = G'_ij - g_i - g_j + mean . mean with
+// G' = X X^T and g = X mean: the Gram kernel then contracts over features (both operands K-major, a CTA owns a
+// 256 x 256 block pair of tokens and a chunk of 64-feature slices) and everything after it runs at size N.
 // Every wait is bounded: the TMA / MMA barriers as in the other tensor-core kernels, the grid barrier by a
 // poll limit after which the kernel raises UNCOMP_STATUS_TIMEOUT and all CTAs leave.
 #include <math.h>
@@ -90,7 +94,11 @@ struct WideTail {
 };
 constexpr int kWSmem = 1024 + kWStages * kWStage + (int)sizeof(WideTail);
 
-// grid (block pairs, token chunks)
+// grid (block pairs, chunks of the contracted dimension).  DUAL = false: blocks of 256 features, contraction over
+// tokens in stages of 64 (operands MN-major); DUAL = true: blocks of 256 tokens, contraction over features in slices
+// of 64 (operands K-major: rows 128 B apart, 8-row groups 1024 B apart, 16 features further = 32 B).
+// N here is the extent of the contracted dimension, chunk its share per CTA (a multiple of 64).
+template <bool DUAL>
 __global__ void __launch_bounds__(kWThreads, 1)
 gram_wide_kernel(const __grid_constant__ CUtensorMap tmap, int N, int nblk, int chunk, float *__restrict__ partials,
                  uint32_t *__restrict__ status) {
@@ -146,12 +154,18 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap tmap, int N, int nblk, int 
                 const uint32_t bar = tc::smem_u32(&T.full[s]);
                 const uint32_t dst = tiles_addr + s * kWStage;
                 tc::mbar_expect_tx(bar, diag ? kWHalf : kWStage);
-#pragma unroll
-                for (int r = 0; r < 4; ++r) tc::tma_load_3d(dst + r * kWRegion, &tmap, bar, I * kWBlock + r * 64, t0 + i * kWTok, 0);
-                if (!diag) {
+                if (DUAL) {      // one box of 64 features x 256 tokens per block
+                    tc::tma_load_3d(dst, &tmap, bar, t0 + i * kWTok, I * kWBlock, 0);
+                    if (!diag) tc::tma_load_3d(dst + kWHalf, &tmap, bar, t0 + i * kWTok, J * kWBlock, 0);
+                } else {
 #pragma unroll
                     for (int r = 0; r < 4; ++r)
-                        tc::tma_load_3d(dst + kWHalf + r * kWRegion, &tmap, bar, J * kWBlock + r * 64, t0 + i * kWTok, 0);
+                        tc::tma_load_3d(dst + r * kWRegion, &tmap, bar, I * kWBlock + r * 64, t0 + i * kWTok, 0);
+                    if (!diag) {
+#pragma unroll
+                        for (int r = 0; r < 4; ++r)
+                            tc::tma_load_3d(dst + kWHalf + r * kWRegion, &tmap, bar, J * kWBlock + r * 64, t0 + i * kWTok, 0);
+                    }
                 }
             }
             if (T.abort) {
@@ -161,10 +175,13 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap tmap, int N, int nblk, int 
         }
     } else if (warp == 5) {
         if (lane == 0) {
-            constexpr uint32_t idesc = tc::idesc_bf16_f32(128, 256, 1, 1);
+            constexpr uint32_t idesc = DUAL ? tc::idesc_bf16_f32(128, 256, 0, 0) : tc::idesc_bf16_f32(128, 256, 1, 1);
             // MN-major, 128-byte swizzle: 64-feature regions kWRegion apart (LBO), 8-token groups 1024 B apart
-            // (SBO); 16 tokens further = 2048 B = +128 in the 16-byte address field
-            const uint64_t base_desc = tc::smem_desc_sw128(tiles_addr, kWRegion, 1024);
+            // (SBO); 16 tokens further = 2048 B = +128 in the 16-byte address field.  K-major: 8-row groups 1024 B
+            // apart, 16 features further = 32 B = +2; the second 128 rows of a block start 16 KB further.
+            constexpr uint32_t kStep = DUAL ? 2u : 128u;
+            constexpr uint32_t kSecondHalf = DUAL ? (uint32_t)((128 * 128) >> 4) : (uint32_t)((2 * kWRegion) >> 4);
+            const uint64_t base_desc = tc::smem_desc_sw128(tiles_addr, DUAL ? 16 : kWRegion, 1024);
             const uint32_t dhi = tc::desc_hi(base_desc);
             bool ok = true;
             for (int i = 0; i < ntiles && ok; ++i) {
@@ -177,9 +194,8 @@ gram_wide_kernel(const __grid_constant__ CUtensorMap tmap, int N, int nblk, int 
 #pragma unroll
                 for (int k = 0; k < kWTok / 16; ++k) {
                     const uint32_t acc = (i > 0 || k > 0) ? 1u : 0u;
-                    tc::mma_f16_ss_lohi(tmem, lo + k * 128, b_lo + k * 128, dhi, idesc, acc);
-                    tc::mma_f16_ss_lohi(tmem + 256, lo + (uint32_t)((2 * kWRegion) >> 4) + k * 128, b_lo + k * 128, dhi, idesc,
-                                        acc);
+                    tc::mma_f16_ss_lohi(tmem, lo + k * kStep, b_lo + k * kStep, dhi, idesc, acc);
+                    tc::mma_f16_ss_lohi(tmem + 256, lo + kSecondHalf + k * kStep, b_lo + k * kStep, dhi, idesc, acc);
                 }
                 tc::mma_commit(tc::smem_u32(&T.empty[s]));
             }
@@ -239,6 +255,49 @@ __global__ void __launch_bounds__(256) wide_assemble_kernel(const float *__restr
     const float v = (float)acc;
     C[(size_t)gi * D + gj] = v;
     C[(size_t)gj * D + gi] = v;
+}
+
+// Token-space variant: C'_ij = G'_ij - g_i - g_j + mm for i, j < N (g = X mean, mm = mean . mean, stored at g[Dt]);
+// rows and columns N .. Dt - 1 only pad the matrix to a multiple of 64 and are zero.
+__global__ void __launch_bounds__(256) wide_assemble_dual_kernel(const float *__restrict__ partials, int pairs, int chunks,
+                                                                int nblk, int Dt, int N, int center,
+                                                                const double *__restrict__ g, float *__restrict__ C) {
+    int I = 0, J = 0;
+    {
+        int rem = blockIdx.x;
+        for (I = 0; I < nblk; ++I) {
+            const int cnt = nblk - I;
+            if (rem < cnt) { J = I + rem; break; }
+            rem -= cnt;
+        }
+    }
+    const int r = blockIdx.y, c = threadIdx.x;
+    const int gi = I * kWBlock + r, gj = J * kWBlock + c;
+    if (gi >= Dt || gj >= Dt || (I == J && r > c)) return;
+    const int mi = r >> 7, m = r & 127;
+    double acc = 0.0;
+    if (gi < N && gj < N) {
+        for (int ch = 0; ch < chunks; ++ch)
+            acc += (double)partials[(((size_t)ch * pairs + blockIdx.x) * 2 + mi) * (128 * kWBlock) + (size_t)m * kWBlock + c];
+        if (center) acc += g[Dt] - g[gi] - g[gj];
+    }
+    const float v = (float)acc;
+    C[(size_t)gi * Dt + gj] = v;
+    C[(size_t)gj * Dt + gi] = v;
+}
+
+// g_i = x_i . mean (a warp per token, fp64) and mean . mean at g[Dt]
+__global__ void __launch_bounds__(256) wide_rowdot_kernel(const __nv_bfloat16 *__restrict__ X, int64_t sN, int N, int D, int Dt,
+                                                         const double *__restrict__ s, double *__restrict__ g) {
+    const int lane = threadIdx.x & 31, row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row > N) return;                                  // warp N computes mean . mean
+    double acc = 0.0;
+    for (int f = lane; f < D; f += 32) {
+        const double m = s[f] / (double)N;
+        acc += (row < N ? (double)__bfloat162float(X[(int64_t)row * sN + f]) : m) * m;
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) g[row < N ? row : Dt] = acc;
 }
 
 // ------------------------------------------------------------------------------------- 4. tridiagonalisation
@@ -493,53 +552,61 @@ __global__ void __launch_bounds__(kSturmThreads) sturm_wide_kernel(const double 
     }
 }
 
-// H_k and erank_k from the k largest eigenvalues (descending) and the trace at lam[k]
-__global__ void wide_entropy_kernel(const double *__restrict__ lam, int k, int norm, float *__restrict__ H_out,
+// H_k and erank_k from the kf largest eigenvalues (descending; eigenvalues kf .. k - 1 are zero) and the trace at
+// lam[kf]
+__global__ void wide_entropy_kernel(const double *__restrict__ lam, int k, int kf, int norm, float *__restrict__ H_out,
                                     float *__restrict__ erank_out, double *__restrict__ spectrum) {
     if (threadIdx.x != 0) return;
     double denom = 0.0;
     if (norm == 0) {
-        for (int i = 0; i < k; ++i) denom += fmax(lam[i], 0.0);
+        for (int i = 0; i < kf; ++i) denom += fmax(lam[i], 0.0);
     } else {
-        denom = lam[k];
+        denom = lam[kf];
     }
     double h = 0.0;
-    for (int i = 0; i < k; ++i) {
+    for (int i = 0; i < kf; ++i) {
         const double pi = denom > 0.0 ? fmax(lam[i], 0.0) / denom : 0.0;
         if (pi > 0.0) h -= pi * log(pi);
     }
     *H_out = (float)h;
     if (erank_out) *erank_out = (float)exp(h);
     if (spectrum)
-        for (int i = 0; i < k; ++i) spectrum[i] = lam[i];
+        for (int i = 0; i < k; ++i) spectrum[i] = i < kf ? lam[i] : 0.0;
 }
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct WideLayout {
+    bool dual;          // token-space path (N < D)
+    int Dt;             // size of the symmetric matrix that is tridiagonalised
     int nblk, pairs, chunk, chunks;
-    size_t off_bar, off_s, off_colpart, off_a, off_e, off_lam, off_p, off_C, off_part, bytes;
+    size_t off_bar, off_s, off_colpart, off_a, off_e, off_lam, off_g, off_p, off_C, off_part, bytes;
 };
 
 WideLayout wide_layout(int N, int D) {
     WideLayout w;
-    w.nblk = (D + kWBlock - 1) / kWBlock;
+    w.dual = N < D;
+    w.Dt = w.dual ? (N + 63) / 64 * 64 : D;
+    if (w.Dt < 128) w.Dt = 128;
+    const int contract = w.dual ? D : N;                     // extent of the contracted dimension
+    w.nblk = (w.Dt + kWBlock - 1) / kWBlock;
     w.pairs = w.nblk * (w.nblk + 1) / 2;
     int chunks = (2 * 148 + w.pairs - 1) / w.pairs;          // about two CTAs' worth of work per SM
-    const int max_chunks = (N + 511) / 512;
+    const int max_chunks = (contract + 511) / 512;
     if (chunks > max_chunks) chunks = max_chunks;
     if (chunks < 1) chunks = 1;
-    w.chunk = (((N + chunks - 1) / chunks) + kWTok - 1) / kWTok * kWTok;
-    w.chunks = (N + w.chunk - 1) / w.chunk;
+    w.chunk = (((contract + chunks - 1) / chunks) + kWTok - 1) / kWTok * kWTok;
+    w.chunks = (contract + w.chunk - 1) / w.chunk;
     size_t o = 0;
     w.off_bar = o;      o = align256(o + 256);
     w.off_s = o;        o = align256(o + (size_t)D * sizeof(double));
     w.off_colpart = o;  o = align256(o + (size_t)kColChunks * D * sizeof(double));
-    w.off_a = o;        o = align256(o + (size_t)D * sizeof(double));
-    w.off_e = o;        o = align256(o + (size_t)D * sizeof(double));
+    w.off_a = o;        o = align256(o + (size_t)w.Dt * sizeof(double));
+    w.off_e = o;        o = align256(o + (size_t)w.Dt * sizeof(double));
     w.off_lam = o;      o = align256(o + (size_t)(kSturmMaxK + 1) * sizeof(double));
-    w.off_p = o;        o = align256(o + (size_t)2 * D * sizeof(float));
-    w.off_C = o;        o = align256(o + (size_t)D * D * sizeof(float));
+    w.off_g = o;        o = align256(o + (size_t)(w.Dt + 1) * sizeof(double));
+    w.off_p = o;        o = align256(o + (size_t)2 * w.Dt * sizeof(float));
+    w.off_C = o;        o = align256(o + (size_t)w.Dt * w.Dt * sizeof(float));
     w.off_part = o;     o = align256(o + (size_t)w.chunks * w.pairs * 2 * 128 * kWBlock * sizeof(float));
     w.bytes = o;
     return w;
@@ -556,6 +623,7 @@ cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const
     double *s = (double *)(scratch + w.off_s), *colpart = (double *)(scratch + w.off_colpart);
     double *a = (double *)(scratch + w.off_a), *e = (double *)(scratch + w.off_e);
     float *pbuf = (float *)(scratch + w.off_p), *C = (float *)(scratch + w.off_C), *part = (float *)(scratch + w.off_part);
+    double *g = (double *)(scratch + w.off_g);
     unsigned *bar = (unsigned *)(scratch + w.off_bar);
     cudaError_t err = cudaMemsetAsync(bar, 0, 256, st);
     if (err != cudaSuccess) return err;
@@ -566,16 +634,26 @@ cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const
         CUtensorMap tmap;
         uint64_t dims[3] = {(uint64_t)D, (uint64_t)N, 1};
         uint64_t str[2] = {(uint64_t)sN * 2, (uint64_t)sN * 2 * (uint64_t)N};
-        uint32_t box[3] = {64, (uint32_t)kWTok, 1};
+        uint32_t box[3] = {64, w.dual ? (uint32_t)kWBlock : (uint32_t)kWTok, 1};
         err = encode_tensor_map(&tmap, d_X, 3, dims, str, box, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B);
         if (err != cudaSuccess) return err;
-        err = cudaFuncSetAttribute(gram_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem);
-        if (err != cudaSuccess) return err;
-        gram_wide_kernel<<<dim3(w.pairs, w.chunks), kWThreads, kWSmem, st>>>(tmap, N, w.nblk, w.chunk, part, d_status);
+        if (w.dual) {
+            err = cudaFuncSetAttribute(gram_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem);
+            if (err != cudaSuccess) return err;
+            gram_wide_kernel<true><<<dim3(w.pairs, w.chunks), kWThreads, kWSmem, st>>>(tmap, D, w.nblk, w.chunk, part, d_status);
+            wide_rowdot_kernel<<<(N + 1 + 7) / 8, 256, 0, st>>>(X, sN, N, D, w.Dt, s, g);
+        } else {
+            err = cudaFuncSetAttribute(gram_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kWSmem);
+            if (err != cudaSuccess) return err;
+            gram_wide_kernel<false><<<dim3(w.pairs, w.chunks), kWThreads, kWSmem, st>>>(tmap, N, w.nblk, w.chunk, part, d_status);
+        }
     }
     {
         ProfScope ps(prof, kSlotWideAssemble, st);
-        wide_assemble_kernel<<<dim3(w.pairs, kWBlock), 256, 0, st>>>(part, w.pairs, w.chunks, w.nblk, D, N, ep.center, s, C);
+        if (w.dual)
+            wide_assemble_dual_kernel<<<dim3(w.pairs, kWBlock), 256, 0, st>>>(part, w.pairs, w.chunks, w.nblk, w.Dt, N, ep.center, g, C);
+        else
+            wide_assemble_kernel<<<dim3(w.pairs, kWBlock), 256, 0, st>>>(part, w.pairs, w.chunks, w.nblk, D, N, ep.center, s, C);
     }
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
@@ -584,25 +662,29 @@ cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const
         int dev = 0, sms = 0, per_sm = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        const size_t smem = (size_t)3 * D * sizeof(float);
+        const int Dt = w.Dt;
+        const size_t smem = (size_t)3 * Dt * sizeof(float);
         err = cudaFuncSetAttribute(tridiag_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
         err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tridiag_wide_kernel, kTriThreads, smem);
         if (err != cudaSuccess) return err;
         if (per_sm < 1) return cudaErrorLaunchOutOfResources;
         int grid = sms;                                          // one CTA per SM: all of them are resident
-        if (grid > D / 8) grid = D / 8;                           // small matrices: fewer CTAs, cheaper barrier
-        int Di = D;
+        if (grid > Dt / 8) grid = Dt / 8;                         // small matrices: fewer CTAs, cheaper barrier
+        int Di = Dt;
         void *args[] = {(void *)&C, (void *)&Di, (void *)&a, (void *)&e, (void *)&pbuf, (void *)&bar, (void *)&d_status};
         err = cudaLaunchCooperativeKernel((const void *)tridiag_wide_kernel, dim3(grid), dim3(kTriThreads), args, smem, st);
         if (err != cudaSuccess) return err;
     }
     {
         ProfScope ps(prof, kSlotWideSturm, st);
-        const int k = ep.k_trunc < D ? ep.k_trunc : D;
+        const int k = ep.k_trunc < D ? ep.k_trunc : D;            // entries of the outputs
+        const int kf = k < w.Dt ? k : w.Dt;                       // eigenvalues the matrix can have; the rest are zero
         double *lam = (double *)(scratch + w.off_lam);
-        sturm_wide_kernel<<<k, kSturmThreads, 0, st>>>(a, e, D, k, ep.max_iters, lam, d_status);
-        wide_entropy_kernel<<<1, 32, 0, st>>>(lam, k, ep.norm, d_entropy, d_erank, d_spectrum);
+        err = cudaMemsetAsync(lam, 0, (size_t)(kSturmMaxK + 1) * sizeof(double), st);
+        if (err != cudaSuccess) return err;
+        sturm_wide_kernel<<<kf, kSturmThreads, 0, st>>>(a, e, w.Dt, kf, ep.max_iters, lam, d_status);
+        wide_entropy_kernel<<<1, 32, 0, st>>>(lam, k, kf, ep.norm, d_entropy, d_erank, d_spectrum);
     }
     return cudaGetLastError();
 }

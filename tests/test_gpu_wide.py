@@ -41,6 +41,10 @@ def _check(ub, X, k, center, norm):
     (1000, 384, 40, 32, 1, 0),      # second block half empty
     (333, 512, 6, 16, 0, 0),        # N < D, uncentred
     (2500, 1024, 64, 64, 1, 1),     # ten block pairs, several token chunks, whole-trace normalisation
+    (700, 1024, 30, 32, 1, 0),      # fewer tokens than features: token-space path, ragged token count, centred
+    (100, 256, 8, 32, 1, 1),        # token-space matrix padded from 100 to 128, whole-trace normalisation
+    (1000, 4096, 50, 64, 1, 0),     # hidden-state width, short prompt
+    (60, 512, 5, 64, 1, 0),         # k_trunc beyond the number of tokens: the missing eigenvalues are zero
 ])
 def test_entropy_wide_parity(N, D, rank, k, center, norm):
     from paper_2410_03090_b200 import binding as ub
