@@ -182,3 +182,19 @@ def test_decode_seed_matches_oracle():
     idx1 = torch.arange(56, 64, dtype=torch.int32, device="cuda")
     off1 = torch.tensor([0, 8], dtype=torch.int64, device="cuda")
     assert float(ub.uncomp_decode_seed(ctx, scores, idx1, off1).abs().max()) == 0.0
+
+
+def test_decode_update_same_bits_twice():
+    from paper_2410_03090_b200 import binding as ub
+    caps = [1500, 700, 2048, 33]
+    results = []
+    for _ in range(2):
+        ctx = ub.Context(ub.make_shape(1, 1, 4, 16, 8192, 128, 32, "bf16"))
+        st = State(1, 1, 4, 16, "bf16", caps, caps, seed=17)
+        q, k, v = st.new_token()
+        p = torch.zeros(sum(caps) + 4, device="cuda")
+        npos = torch.tensor([st.new_pos], dtype=torch.int32, device="cuda")
+        ub.uncomp_decode_update(ctx, q, k, v, npos, st.offsets, st.lens, 2048, st.Kc, st.Vc, st.pos, st.cum, p=p)
+        torch.cuda.synchronize()
+        results.append((p, st.cum.clone(), st.pos.clone(), st.Kc.clone()))
+    assert all(torch.equal(a, b) for a, b in zip(*results))

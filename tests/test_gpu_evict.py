@@ -70,3 +70,18 @@ def test_evict_hidden_rejections():
     with pytest.raises(ub.UncompError) as ei:
         ub.uncomp_evict_hidden(ctx, q, K, X[:, :, :60].contiguous(), 10)     # rows of 120 bytes
     assert ei.value.code == ub.UNCOMP_E_ALIGN
+
+
+def test_evict_hidden_same_bits_twice():
+    from paper_2410_03090_b200 import binding as ub
+    g = torch.Generator(device="cuda").manual_seed(9)
+    q = torch.randn(2, 32, 128, generator=g, device="cuda").to(torch.bfloat16)
+    K = torch.randn(2, 8, 5000, 128, generator=g, device="cuda").to(torch.bfloat16)
+    X = torch.randn(2, 5000, 256, generator=g, device="cuda").to(torch.bfloat16)
+    ctx = ub.Context(ub.make_shape(2, 1, 8, 32, 5000, 128, 1, "bf16"))
+    runs = []
+    for _ in range(2):
+        sc = torch.empty(2, 4999, device="cuda")
+        idx, Xo = ub.uncomp_evict_hidden(ctx, q, K, X, 1234, scores=sc)
+        runs.append((sc.clone(), idx.clone(), Xo.clone()))
+    assert all(torch.equal(a, b) for a, b in zip(*runs))
