@@ -12,6 +12,8 @@
 //      kept position its output slot, so the kept positions come out ascending, and among scores equal to
 //      T the lowest positions win.  The window positions follow.
 // Counting is integer work: the result does not depend on the order in which threads run.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace uncomp {
@@ -142,11 +144,139 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float *_
     }
 }
 
+// The same selection with a unit spread over a cluster of 8 CTAs, for calls with few units (a layer of one sequence,
+// the hidden-state eviction with one unit per sequence), where one CTA per unit would leave most SMs idle.  CTA r of
+// the cluster owns the r-th eighth of the positions; histograms and counts are combined through distributed shared
+// memory by CTA 0 and read back by the others.  The result is identical to the single-CTA kernel.
+constexpr int kSelCluster = 8;
+
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
+pool_select_cluster_kernel(const float *__restrict__ raw, float *__restrict__ pooled, int P, int w, int pool_kernel,
+                           int pool_mode, const int32_t *__restrict__ budgets, const int64_t *__restrict__ offsets,
+                           int32_t *__restrict__ indices, uint32_t *__restrict__ status) {
+    namespace cg = cooperative_groups;
+    __shared__ SelSmem S;
+    __shared__ int slice_gt, slice_eq;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int u = blockIdx.x / kSelCluster, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const float *r = raw + (size_t)u * P;
+    float *s = pooled + (size_t)u * P;
+    // this CTA's positions: a multiple of 1024 per CTA, so that warps own aligned segments of 32
+    const int per = ((P + kSelCluster - 1) / kSelCluster + kSelThreads - 1) / kSelThreads * kSelThreads;
+    const int p0 = min(P, rank * per), p1 = min(P, p0 + per);
+
+    const int half = pool_kernel >> 1;
+    for (int j = p0 + tid; j < p1; j += kSelThreads) {
+        const int lo = max(0, j - half), hi = min(P - 1, j + half);
+        float acc = pool_mode ? 0.f : r[lo];
+        for (int t = lo; t <= hi; ++t) acc = pool_mode ? acc + r[t] : fmaxf(acc, r[t]);
+        s[j] = pool_mode ? acc / (float)(hi - lo + 1) : acc;
+    }
+    int budget = budgets[u];
+    if (budget < w || budget > P + w) {
+        if (tid == 0 && rank == 0) atomicOr(status, UNCOMP_STATUS_BOUNDS);
+        budget = min(max(budget, w), P + w);
+    }
+    const int k = budget - w;
+    int32_t *out = indices + offsets[u];
+    if (rank == 0)
+        for (int i = tid; i < w; i += kSelThreads) out[k + i] = P + i;
+    if (k == 0) return;   // uniform over the cluster
+    __syncthreads();      // this CTA reads only the pooled scores it wrote itself
+
+    SelSmem *S0 = cluster.map_shared_rank(&S, 0);
+    uint32_t prefix = 0;
+    int kr = k;
+    if (k < P) {
+#pragma unroll 1
+        for (int pass = 0; pass < 3; ++pass) {
+            const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+            const int nbits = pass == 2 ? 10 : 11;
+            const int nbins = 1 << nbits;
+            const uint32_t himask = pass == 0 ? 0u : (0xffffffffu << (shift + nbits));
+            for (int b = tid; b < 2048; b += kSelThreads) S.hist[b] = 0;
+            __syncthreads();
+            for (int j = p0 + tid; j < p1; j += kSelThreads) {
+                const uint32_t v = ordered_bits(s[j]);
+                if ((v & himask) == prefix) atomicAdd(&S.hist[(v >> shift) & (nbins - 1)], 1);
+            }
+            cluster.sync();                       // every CTA's histogram is complete
+            if (rank == 0) {
+                for (int b = tid; b < nbins; b += kSelThreads) {
+                    int sum = S.hist[b];
+                    for (int c = 1; c < kSelCluster; ++c) sum += cluster.map_shared_rank(&S, c)->hist[b];
+                    S.hist[b] = sum;              // only this thread reads or writes bin b of CTA 0 here
+                }
+                __syncthreads();
+                find_bin(S, nbins, kr, tid);
+            }
+            cluster.sync();                       // bin and count above it are published by CTA 0
+            prefix |= (uint32_t)S0->bin << shift;
+            kr -= S0->above;
+            cluster.sync();                       // all have read them before the next pass clears the histograms
+        }
+    }
+    const uint32_t T = k < P ? prefix : 0u;
+    const int need_eq = k < P ? kr : P;
+
+    // ordered compaction: counts of the lower CTAs first, then of the lower warps of this CTA
+    const int seg = per / kSelWarps;              // a multiple of 32
+    const int j0 = min(p1, p0 + wid * seg), j1 = min(p1, j0 + seg);
+    int cg_ = 0, ce = 0;
+    for (int j = j0 + lane; j < j1; j += 32) {
+        const uint32_t v = ordered_bits(s[j]);
+        cg_ += v > T;
+        ce += v == T;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        cg_ += __shfl_xor_sync(0xffffffffu, cg_, o);
+        ce += __shfl_xor_sync(0xffffffffu, ce, o);
+    }
+    if (lane == 0) { S.warp_gt[wid] = cg_; S.warp_eq[wid] = ce; }
+    __syncthreads();
+    if (tid == 0) {
+        int a = 0, b = 0;
+        for (int x = 0; x < kSelWarps; ++x) { a += S.warp_gt[x]; b += S.warp_eq[x]; }
+        slice_gt = a;
+        slice_eq = b;
+    }
+    cluster.sync();
+    int gt_run = 0, eq_run = 0;
+    for (int c = 0; c < rank; ++c) {
+        gt_run += *cluster.map_shared_rank(&slice_gt, c);
+        eq_run += *cluster.map_shared_rank(&slice_eq, c);
+    }
+    for (int x = 0; x < wid; ++x) { gt_run += S.warp_gt[x]; eq_run += S.warp_eq[x]; }
+    const unsigned lt = (1u << lane) - 1u;
+    for (int jb = j0; jb < j1; jb += 32) {
+        const int j = jb + lane;
+        const uint32_t v = j < j1 ? ordered_bits(s[j]) : 0u;
+        const bool gt = j < j1 && v > T;
+        const bool eq = j < j1 && v == T;
+        const unsigned mg = __ballot_sync(0xffffffffu, gt), me = __ballot_sync(0xffffffffu, eq);
+        const int gtb = gt_run + __popc(mg & lt);
+        const int eqb = eq_run + __popc(me & lt);
+        if (gt || (eq && eqb < need_eq)) out[gtb + min(eqb, need_eq)] = j;
+        gt_run += __popc(mg);
+        eq_run += __popc(me);
+    }
+    cluster.sync();       // no CTA leaves while another may still read its shared memory
+}
+
 cudaError_t launch_pool_select(const Plan &p, const float *d_raw, float *d_pooled, int pool_kernel, int pool_mode,
                                const int32_t *d_budgets, const int64_t *d_offsets, int32_t *d_indices,
                                uint32_t *d_status, cudaStream_t st) {
-    pool_select_kernel<<<p.units, kSelThreads, 0, st>>>(d_raw, d_pooled, p.prefix, p.shape.w, pool_kernel, pool_mode,
-                                                        d_budgets, d_offsets, d_indices, d_status);
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (p.units * kSelCluster <= 2 * sms && p.prefix >= 4096)      // few units: a cluster of CTAs per unit
+        pool_select_cluster_kernel<<<p.units * kSelCluster, kSelThreads, 0, st>>>(
+            d_raw, d_pooled, p.prefix, p.shape.w, pool_kernel, pool_mode, d_budgets, d_offsets, d_indices, d_status);
+    else
+        pool_select_kernel<<<p.units, kSelThreads, 0, st>>>(d_raw, d_pooled, p.prefix, p.shape.w, pool_kernel, pool_mode,
+                                                            d_budgets, d_offsets, d_indices, d_status);
     return cudaGetLastError();
 }
 

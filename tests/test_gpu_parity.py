@@ -404,3 +404,26 @@ def test_scores_may_stay_in_the_workspace():
     torch.cuda.synchronize()
     assert ub.uncomp_status(ctx) == 0 and torch.equal(idx_a, idx_b)
     parity.check_select(wl, scores, b, o, idx_b, range(wl.units))
+
+
+@pytest.mark.parametrize("units,N,w,budget", [(1, 9000, 32, 700), (4, 32768, 64, 5000), (8, 4200, 8, 4100), (3, 20001, 16, 16)])
+def test_select_with_few_units_takes_the_cluster_kernel_and_matches_oracle(units, N, w, budget):
+    """Few units and a long prefix: the selection runs as a cluster of CTAs per unit; same answer, bit for bit."""
+    import oracle
+    from paper_2410_03090_b200 import binding as ub
+    g = torch.Generator(device="cuda").manual_seed(units * 7 + N)
+    K = torch.randn(1, 1, units, N, 128, generator=g, device="cuda").to(torch.bfloat16)
+    Qw = torch.randn(1, 1, units, w, 128, generator=g, device="cuda").to(torch.bfloat16)
+    dup = torch.arange(0, N - 1, 7, device="cuda")
+    K[:, :, :, dup] = K[:, :, :, dup + 1]                      # duplicated keys: exact score ties
+    ctx = ub.Context(ub.make_shape(1, 1, units, units, N, 128, w, "bf16"))
+    budgets = torch.full((1, 1, units), budget, dtype=torch.int32, device="cuda")
+    offsets = (torch.arange(units + 1, device="cuda") * budget).to(torch.int64)
+    scores = torch.empty(1, 1, units, N - w, device="cuda")
+    idx = torch.empty(units * budget, dtype=torch.int32, device="cuda")
+    ub.uncomp_score_select(ctx, Qw, K, budgets, offsets, units * budget, 7, 0, 0.0, scores, idx)
+    torch.cuda.synchronize()
+    assert ub.uncomp_status(ctx) == 0
+    for u in range(units):
+        want = oracle.select(scores[0, 0, u].double().cpu().numpy(), w, budget)
+        np.testing.assert_array_equal(idx[u * budget:(u + 1) * budget].cpu().numpy(), want)
