@@ -863,20 +863,28 @@ def main():
         h2d = sum(t.numel() * t.element_size() for t in (hK, hV, hQ))
         d2h = sum(t.numel() * t.element_size() for t in outs)
 
-        # The results of a step go back on a second stream, so that their device-to-host copy overlaps the
-        # host-to-device copy of the next step's inputs (the link is full duplex); the next pass waits for that copy
-        # before it overwrites the outputs.  Every step still moves all of its inputs and all of its results.
-        out_stream = torch.cuda.Stream(device=dev)
-        done_pass, done_out = torch.cuda.Event(), torch.cuda.Event()
+        # Three streams.  The inputs arrive on the main stream, keys and window queries first; the pass runs on a
+        # second stream and starts as soon as those two are there, so that everything but the final gather overlaps the
+        # copy of the values; the results go back on a third stream and overlap the next step's input copies (the link
+        # is full duplex).  Every step still moves all of its inputs and all of its results.
+        pass_stream, out_stream = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        have_kq, have_v, done_pass, done_out = (torch.cuda.Event() for _ in range(4))
 
         def e2e_step(first=False):
-            dK.copy_(hK, non_blocking=True)
-            dV.copy_(hV, non_blocking=True)
-            dQ.copy_(hQ, non_blocking=True)
             if not first:
-                stream.wait_event(done_out)
-            cp.run(dK, dV, dQ)
-            done_pass.record(stream)
+                stream.wait_event(done_pass)          # the last pass no longer reads the input buffers
+            dK.copy_(hK, non_blocking=True)
+            dQ.copy_(hQ, non_blocking=True)
+            have_kq.record(stream)
+            dV.copy_(hV, non_blocking=True)
+            have_v.record(stream)
+            pass_stream.wait_event(have_kq)
+            if not first:
+                pass_stream.wait_event(done_out)      # the last results have left the output buffers
+            cp.score(dK, dQ, stream=pass_stream)
+            pass_stream.wait_event(have_v)
+            cp.compact(dK, dV, stream=pass_stream)
+            done_pass.record(pass_stream)
             out_stream.wait_event(done_pass)
             with torch.cuda.stream(out_stream):
                 for h, t in zip(houts, outs):

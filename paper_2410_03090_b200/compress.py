@@ -48,16 +48,27 @@ class CompressionPass:
             Vc=torch.empty(wl.total_rows, wl.d, dtype=wl.torch_dtype, device=dev),
         )
 
-    def run(self, K: torch.Tensor, V: torch.Tensor, Qw: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
-            eps: float = 0.0, dn: int = 0, n_last: int = 0, scope: int = 0) -> PassOutput:
+    def score(self, K: torch.Tensor, Qw: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
+              eps: float = 0.0, dn: int = 0, n_last: int = 0, scope: int = 0) -> PassOutput:
+        """Everything that needs only the keys and the window queries: entropy, budgets, scores, kept positions."""
         wl, o, ctx = self.wl, self.out, self.ctx
         ub.uncomp_entropy(ctx, K, wl.k_trunc, 1, 0, 0, o.entropy, o.erank, None, stream, Qw=Qw if self.fused else None)
         ub.uncomp_assign_budgets(ctx, o.erank, wl.avg_budget, wl.M, wl.n_max, scope, eps, dn, n_last,
                                  o.budgets, o.offsets, o.layer_group, o.layer_ctx, stream)
         ub.uncomp_score_select(ctx, Qw, K, o.budgets, o.offsets, wl.total_rows, wl.pool_kernel, wl.pool_mode, 0.0,
                                o.scores, o.indices, stream)
-        ub.uncomp_compact(ctx, K, V, o.indices, o.offsets, wl.total_rows, o.Kc, o.Vc, stream)
         return o
+
+    def compact(self, K: torch.Tensor, V: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> PassOutput:
+        """The gather of the kept K and V rows; the only step that touches the values."""
+        wl, o = self.wl, self.out
+        ub.uncomp_compact(self.ctx, K, V, o.indices, o.offsets, wl.total_rows, o.Kc, o.Vc, stream)
+        return o
+
+    def run(self, K: torch.Tensor, V: torch.Tensor, Qw: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
+            eps: float = 0.0, dn: int = 0, n_last: int = 0, scope: int = 0) -> PassOutput:
+        self.score(K, Qw, stream, eps, dn, n_last, scope)
+        return self.compact(K, V, stream)
 
     def status(self, stream=None) -> int:
         return ub.uncomp_status(self.ctx, stream)
