@@ -311,21 +311,33 @@ def run_hidden(args):
         houts = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
         dq, dK, dX = torch.empty_like(hq, device=dev), torch.empty_like(hK, device=dev), torch.empty_like(X)
 
-        def e2e_step():
+        # the results return on a second stream and overlap the next step's input copies (full-duplex link); the next
+        # step waits for them before it overwrites the outputs
+        out_stream = torch.cuda.Stream(device=dev)
+        done_step, done_out = torch.cuda.Event(), torch.cuda.Event()
+
+        def e2e_step(first=False):
             dq.copy_(hq, non_blocking=True)
             dK.copy_(hK, non_blocking=True)
             dX.copy_(hX, non_blocking=True)
+            if not first:
+                stream.wait_event(done_out)
             step(dq, dK, dX)
-            for h, t in zip(houts, outs):
-                h.copy_(t, non_blocking=True)
+            done_step.record(stream)
+            out_stream.wait_event(done_step)
+            with torch.cuda.stream(out_stream):
+                for h, t in zip(houts, outs):
+                    h.copy_(t, non_blocking=True)
+                done_out.record(out_stream)
 
-        e2e_step()
+        e2e_step(first=True)
         torch.cuda.synchronize()
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(args.e2e_steps):
             e2e_step()
+        stream.wait_event(done_out)
         e1.record(stream)
         torch.cuda.synchronize()
         barrier()
