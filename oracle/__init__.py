@@ -47,6 +47,8 @@ _lib.oracle_majority_vote.argtypes = [_dp, C.c_int, C.c_int, C.c_int, C.c_int, C
 _lib.oracle_majority_vote.restype = C.c_int
 _lib.oracle_decode_seed.argtypes = [_dp, C.c_int, _i32p, C.c_int, _dp]
 _lib.oracle_decode_seed.restype = None
+_lib.oracle_retrieval_layer.argtypes = [_dp, C.c_int, C.c_int, _dp]
+_lib.oracle_retrieval_layer.restype = C.c_int
 _lib.oracle_pool.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _dp]
 _lib.oracle_pool.restype = None
 _lib.oracle_select.argtypes = [_dp, C.c_int, C.c_int, C.c_int, _i32p]
@@ -270,3 +272,11 @@ def decode_seed(score, idx) -> np.ndarray:
     cum = np.empty(len(idx), dtype=np.float64)
     _lib.oracle_decode_seed(_p(score, _dp), len(score), _p(idx, _i32p), len(idx), _p(cum, _dp))
     return cum
+
+
+def retrieval_layer(values):
+    """(layer, increase [L - 1]) for per-head values [L, H]: the layer after the largest rise of the layer mean."""
+    values = _f64(values)
+    L, H = values.shape
+    inc = np.empty(L - 1, dtype=np.float64)
+    return int(_lib.oracle_retrieval_layer(_p(values, _dp), L, H, _p(inc, _dp))), inc

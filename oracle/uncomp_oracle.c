@@ -542,3 +542,32 @@ void oracle_decode_seed(const double *score, int P, const int32_t *idx, int n, d
         if (idx[t] < P && (!any || score[idx[t]] > top)) { top = score[idx[t]]; any = 1; }
     for (int t = 0; t < n; ++t) cum[t] = idx[t] < P ? score[idx[t]] : top;
 }
+
+
+/* ----------------------------------------------------------------------------------------------
+ * Retrieval layer (Section 3.3.2, "Retrieval Layer": the layer with the maximum entropy increase).
+ * values is [L, H] (the truncated entropy, or the effective rank, of every head; e.g. the averaged
+ * values of the preparation stage).  With e_l the mean over the H heads of layer l, increase[l] =
+ * e_{l+1} - e_l for l = 0 .. L-2 and the retrieval layer is l* + 1 for the first l* that attains the
+ * largest increase: the layer whose token matrix gained the most over its predecessor.  L >= 2.
+ * Reading: the paper names the criterion only; taking the layer AFTER the jump, the mean over heads as
+ * the layer's value and the earliest layer on a tie are this implementation's choices.  The merging
+ * of that layer's parameters with the last layer's is a change of model weights and not part of this.
+ * ---------------------------------------------------------------------------------------------- */
+int oracle_retrieval_layer(const double *values, int L, int H, double *increase)
+{
+    int best = 0;
+    double prev = 0.0, best_inc = 0.0;
+    for (int l = 0; l < L; ++l) {
+        double e = 0.0;
+        for (int h = 0; h < H; ++h) e += values[(size_t)l * H + h];
+        e /= (double)H;
+        if (l > 0) {
+            const double inc = e - prev;
+            if (increase) increase[l - 1] = inc;
+            if (l == 1 || inc > best_inc) { best_inc = inc; best = l; }
+        }
+        prev = e;
+    }
+    return best;
+}

@@ -82,3 +82,23 @@ def test_majority_vote_invariants():
         # the order of the samples does not matter
         v2, l2 = oracle.majority_vote(e[::-1], 4, scope)
         np.testing.assert_array_equal(v2, votes)
+
+
+def test_retrieval_layer_worked_cases():
+    # layer means 4, 3, 5, 5.5, 2: rises of -1, +2, +0.5, -3.5 -> the layer after the +2 rise is layer 2
+    v = np.array([[4.0, 4.0], [2.0, 4.0], [6.0, 4.0], [5.0, 6.0], [1.0, 3.0]])
+    layer, inc = oracle.retrieval_layer(v)
+    assert layer == 2
+    np.testing.assert_allclose(inc, [-1.0, 2.0, 0.5, -3.5], rtol=1e-15)
+    # equal rises: the earliest layer;  monotone decrease: the smallest drop wins;  two layers: layer 1
+    assert oracle.retrieval_layer(np.array([[0.0], [1.0], [2.0], [3.0]]))[0] == 1
+    assert oracle.retrieval_layer(np.array([[9.0], [5.0], [4.5], [1.0]]))[0] == 2
+    assert oracle.retrieval_layer(np.array([[3.0, 1.0], [0.0, 0.0]]))[0] == 1
+    # against numpy on random values
+    r = np.random.default_rng(4)
+    for _ in range(50):
+        v = r.standard_normal((int(r.integers(2, 40)), int(r.integers(1, 9))))
+        layer, inc = oracle.retrieval_layer(v)
+        m = v.mean(axis=1)
+        np.testing.assert_allclose(inc, np.diff(m), rtol=1e-12, atol=1e-15)
+        assert layer == int(np.argmax(inc)) + 1
