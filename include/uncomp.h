@@ -377,6 +377,21 @@ int uncomp_entropy_wide(uncomp_ctx *ctx, const void *d_X, int32_t count, int64_t
                         int32_t N, int32_t D, const uncomp_entropy_params *params, void *d_scratch, size_t scratch_bytes,
                         float *d_entropy, float *d_erank, double *d_spectrum, void *stream);
 
+/* ---------------------------------------------------------------------------------------------------
+ * uncomp_retrieval_layer -- Section 3.3.2 "Retrieval Layer": the retrieval layer is chosen as the layer of
+ * maximum entropy increase.  d_values [L, H] holds a per-head value (the truncated entropy or the
+ * effective rank, of one input or averaged by uncomp_prepare_groups); with e_l its mean over the heads of
+ * layer l (fp64, head order), increase[l] = e_{l+1} - e_l and *d_layer = l* + 1 for the first l* with the
+ * largest increase.  Readings: the layer AFTER the jump is reported, a tie goes to the earliest layer.
+ * The paper then merges that layer's parameters with the last layer's by averaging; that is a change of
+ * model weights and outside this library.
+ *
+ * d_values    in   [L, H] float (L, H of the context's shape; L >= 2, L <= 4096)
+ * d_layer     out  [1] int32
+ * d_increase  out  [L - 1] float; may be NULL
+ * ------------------------------------------------------------------------------------------------- */
+int uncomp_retrieval_layer(uncomp_ctx *ctx, const float *d_values, int32_t *d_layer, float *d_increase, void *stream);
+
 /* Synchronise `stream`, copy the status word to *host_bits and clear it on the device.  The only call
  * that waits for the device. */
 int uncomp_status(uncomp_ctx *ctx, void *stream, uint32_t *host_bits);

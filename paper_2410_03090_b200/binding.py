@@ -87,6 +87,8 @@ def _load() -> C.CDLL:
     lib.uncomp_entropy_wide.restype = C.c_int
     lib.uncomp_entropy_wide.argtypes = [vp, vp, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
                                         C.POINTER(uncomp_entropy_params), vp, C.c_size_t, fp, fp, dp, vp]
+    lib.uncomp_retrieval_layer.restype = C.c_int
+    lib.uncomp_retrieval_layer.argtypes = [vp, fp, i32p, fp, vp]
     lib.uncomp_prepare_groups.restype = C.c_int
     lib.uncomp_prepare_groups.argtypes = [vp, fp, C.c_int32, C.c_int32, C.c_int32, fp, i32p, i32p, i32p, vp]
     lib.uncomp_decode_seed.restype = C.c_int
@@ -304,6 +306,16 @@ def uncomp_entropy_wide(ctx: Context, X: torch.Tensor, k_trunc: int = 32, center
                                    _ptr(scratch), scratch.numel(), _ptr(ent), _ptr(er), _ptr(spec), _stream(stream)),
            "uncomp_entropy_wide")
     return (ent, er, spec) if spectrum else (ent, er)
+
+
+def uncomp_retrieval_layer(ctx: Context, values: torch.Tensor, stream=None):
+    """values [L, H] float32 -> (layer int32 [1], increase float32 [L - 1])."""
+    L = values.shape[0]
+    layer = torch.empty(1, dtype=torch.int32, device=values.device)
+    inc = torch.empty(L - 1, dtype=torch.float32, device=values.device)
+    _check(lib.uncomp_retrieval_layer(ctx.handle, _ptr(values), _ptr(layer), _ptr(inc), _stream(stream)),
+           "uncomp_retrieval_layer")
+    return layer, inc
 
 
 def uncomp_prepare_groups(ctx: Context, erank: torch.Tensor, M: int, scope: int = 0, stream=None):

@@ -418,6 +418,16 @@ int uncomp_decode_update(uncomp_ctx *ctx, const void *d_qnew, const void *d_knew
     return UNCOMP_OK;
 }
 
+int uncomp_retrieval_layer(uncomp_ctx *ctx, const float *d_values, int32_t *d_layer, float *d_increase, void *stream) {
+    if (!ctx || !d_values || !d_layer) return UNCOMP_E_NULL;
+    const uncomp_shape &s = ctx->plan.shape;
+    if (s.L < 2) return UNCOMP_E_SHAPE;
+    if (s.L > 4096) return UNCOMP_E_LIMIT;
+    cudaError_t e = launch_retrieval_layer(d_values, s.L, s.H, d_layer, d_increase, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return UNCOMP_OK;
+}
+
 int uncomp_prepare_groups(uncomp_ctx *ctx, const float *d_erank, int32_t S, int32_t M, int32_t scope, float *d_mean,
                           int32_t *d_group_mean, int32_t *d_votes, int32_t *d_group_vote, void *stream) {
     if (!ctx || !d_erank || !d_mean || !d_group_mean || !d_votes || !d_group_vote) return UNCOMP_E_NULL;

@@ -115,6 +115,8 @@ cudaError_t launch_decode_update(const Plan &p, const void *d_q, const void *d_k
                                  int protect, float scale, void *d_Kc, void *d_Vc, int32_t *d_pos, float *d_cum,
                                  float *d_p, int32_t *d_evicted, float *d_logits, float *d_stats, void *d_partial,
                                  float *d_new_cum, uint32_t *d_status, Profiler *prof, cudaStream_t st);
+cudaError_t launch_retrieval_layer(const float *d_values, int L, int H, int32_t *d_layer, float *d_increase,
+                                   cudaStream_t st);
 cudaError_t launch_prepare_groups(const float *d_erank, int S, int L, int H, int M, int scope, float *d_mean,
                                   int32_t *d_group_mean, int32_t *d_votes, int32_t *d_group_vote, Profiler *prof,
                                   cudaStream_t st);

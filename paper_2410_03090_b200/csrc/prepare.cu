@@ -70,7 +70,37 @@ __global__ void __launch_bounds__(kPrepThreads) prepare_finish_kernel(const floa
     for (int i = threadIdx.x; i < n; i += kPrepThreads)
         group_mean[(size_t)set * n + i] = group_of_rank(rank_in_set(vals, n, i), n, M);
 }
+// Retrieval layer (paper Section 3.3.2, "Retrieval Layer"): the layer after the largest rise of the layer mean.
+// One CTA: a thread per layer forms the mean over heads in fp64 (head order), thread 0 scans the rises in layer order.
+__global__ void __launch_bounds__(kPrepThreads) retrieval_layer_kernel(const float *__restrict__ values, int L, int H,
+                                                                      int32_t *__restrict__ layer,
+                                                                      float *__restrict__ increase) {
+    extern __shared__ double lmean[];
+    for (int l = threadIdx.x; l < L; l += kPrepThreads) {
+        double e = 0.0;
+        for (int h = 0; h < H; ++h) e += (double)values[(size_t)l * H + h];
+        lmean[l] = e / (double)H;
+    }
+    __syncthreads();
+    for (int l = threadIdx.x; l + 1 < L; l += kPrepThreads)
+        if (increase) increase[l] = (float)(lmean[l + 1] - lmean[l]);
+    if (threadIdx.x == 0) {
+        int best = 1;
+        double best_inc = lmean[1] - lmean[0];
+        for (int l = 2; l < L; ++l) {
+            const double inc = lmean[l] - lmean[l - 1];
+            if (inc > best_inc) { best_inc = inc; best = l; }
+        }
+        *layer = best;
+    }
+}
 }  // namespace
+
+cudaError_t launch_retrieval_layer(const float *d_values, int L, int H, int32_t *d_layer, float *d_increase,
+                                   cudaStream_t st) {
+    retrieval_layer_kernel<<<1, kPrepThreads, (size_t)L * sizeof(double), st>>>(d_values, L, H, d_layer, d_increase);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_prepare_groups(const float *d_erank, int S, int L, int H, int M, int scope, float *d_mean,
                                   int32_t *d_group_mean, int32_t *d_votes, int32_t *d_group_vote, Profiler *prof,

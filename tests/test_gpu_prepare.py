@@ -45,3 +45,19 @@ def test_prepare_groups_rejections():
     assert ei.value.code == ub.UNCOMP_E_PARAM
     mean, gm, votes, gv = ub.uncomp_prepare_groups(ctx, e, 32, 1)        # all equal: rank = index
     assert torch.equal(gm.cpu().ravel(), torch.arange(32, dtype=torch.int32))
+
+
+@pytest.mark.parametrize("L,H", [(32, 8), (2, 1), (80, 8), (300, 3)])
+def test_retrieval_layer_parity(L, H):
+    from paper_2410_03090_b200 import binding as ub
+    g = torch.Generator(device="cuda").manual_seed(L * 13 + H)
+    v = (torch.randn(L, H, generator=g, device="cuda") * 2 + 10).round(decimals=1).contiguous()
+    if L > 4:
+        v[3] = v[1]
+        v[4] = v[2]                      # the rise 1 -> 2 occurs twice: the earlier one must win if it is the largest
+    ctx = ub.Context(ub.make_shape(1, L, H, H, 256, 128, 8, "bf16"))
+    layer, inc = ub.uncomp_retrieval_layer(ctx, v)
+    torch.cuda.synchronize()
+    want, winc = oracle.retrieval_layer(v.double().cpu().numpy())
+    assert int(layer[0]) == want
+    np.testing.assert_allclose(inc.cpu().numpy(), winc, rtol=1e-6, atol=1e-7)
