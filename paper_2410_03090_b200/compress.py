@@ -72,3 +72,42 @@ class CompressionPass:
 
     def status(self, stream=None) -> int:
         return ub.uncomp_status(self.ctx, stream)
+
+
+def eviction_plan(layer_group, layer_ctx):
+    """Where the prefill evicts hidden states (paper Section 3.3.2; Algorithm 2, "compress hidden states"): host
+    logic over the `layer_group` / `layer_ctx` rows of one sequence as `uncomp_assign_budgets` writes them.
+    Returns [(layer, n_keep)]: before layer `layer` (the first of a new layer group) the hidden states are cut to
+    the `n_keep` positions with the highest last-token attention of layer `layer - 1` (`uncomp_evict_hidden`).
+    A group whose context is not smaller than what is still there needs no call and is left out."""
+    groups = [int(g) for g in layer_group]
+    ctx = [int(c) for c in layer_ctx]
+    plan, current = [], ctx[0] if ctx else 0
+    for l in range(1, len(groups)):
+        if groups[l] != groups[l - 1] and ctx[l] < current:
+            plan.append((l, ctx[l]))
+            current = ctx[l]
+    return plan
+
+
+class DecodeCache:
+    """The ragged per-head cache after a prefill pass plus what the decode-time update needs (positions, cumulative
+    scores, fill levels); `step` runs one `uncomp_decode_update` in place."""
+
+    def __init__(self, cp: CompressionPass, out: Optional[PassOutput] = None):
+        o = cp.out if out is None else out
+        self.ctx, self.wl = cp.ctx, cp.wl
+        self.offsets = o.offsets
+        self.Kc, self.Vc = o.Kc, o.Vc
+        self.pos = o.indices.clone()
+        self.lens = o.budgets.reshape(-1).clone()
+        self.cum = ub.uncomp_decode_seed(cp.ctx, o.scores, o.indices, o.offsets)
+        self.max_cap = int(self.lens.max())
+        self.evicted = torch.empty(self.wl.units, dtype=torch.int32, device=self.Kc.device)
+
+    def step(self, qnew: torch.Tensor, knew: torch.Tensor, vnew: torch.Tensor, new_pos: torch.Tensor, protect: int = 1,
+             stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        """qnew [B, L, Hq, d], knew / vnew [B, L, H, d], new_pos [B] int32; returns the evicted positions [units]."""
+        ub.uncomp_decode_update(self.ctx, qnew, knew, vnew, new_pos, self.offsets, self.lens, self.max_cap, self.Kc,
+                                self.Vc, self.pos, self.cum, protect=protect, evicted=self.evicted, stream=stream)
+        return self.evicted

@@ -79,3 +79,13 @@ def test_kernel_specs_cover_every_profiled_kernel():
     # algorithmic work of the c3 pass: 0.275 TFLOP of Gram, 2.57 GB of bytes
     assert abs(specs["gram"][1] - 0.2749) < 1e-3
     assert abs(synth.WORKLOADS["c3"].algorithmic_bytes() / 1e9 - 2.5695) < 1e-3
+
+
+def test_eviction_plan_host_logic():
+    sys.path.insert(0, ROOT)
+    from paper_2410_03090_b200.compress import eviction_plan
+    # three groups: full context, then two cuts; a boundary into a group that is not smaller needs no call
+    assert eviction_plan([0, 0, 1, 1, 1, 2, 2], [4096, 4096, 1536, 1536, 1536, 1024, 1024]) == [(2, 1536), (5, 1024)]
+    assert eviction_plan([0, 0, 0], [900, 900, 900]) == []
+    assert eviction_plan([0, 1, 2], [500, 500, 300]) == [(2, 300)]
+    assert eviction_plan([], []) == []

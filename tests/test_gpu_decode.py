@@ -198,3 +198,28 @@ def test_decode_update_same_bits_twice():
         torch.cuda.synchronize()
         results.append((p, st.cum.clone(), st.pos.clone(), st.Kc.clone()))
     assert all(torch.equal(a, b) for a, b in zip(*results))
+
+
+def test_decode_cache_wrapper_runs_prefill_then_decode():
+    from paper_2410_03090_b200 import synth
+    from paper_2410_03090_b200.compress import CompressionPass, DecodeCache
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=2048, L=2)
+    K, V, Qw = synth.generate(wl, "cuda")
+    cp = CompressionPass(wl, "cuda")
+    cp.run(K, V, Qw)
+    cache = DecodeCache(cp)
+    offs = cache.offsets.cpu().numpy()
+    for t in range(3):
+        pos_before = cache.pos.clone()
+        npos = torch.full((wl.B,), wl.N + t, dtype=torch.int32, device="cuda")
+        ev = cache.step(Qw[:, :, :, -1 - t, :].contiguous(), K[:, :, :, -1 - t, :].contiguous(),
+                        V[:, :, :, -1 - t, :].contiguous(), npos)
+        torch.cuda.synchronize()
+        assert cp.status() == 0
+        changed = (cache.pos != pos_before).cpu().numpy()
+        assert (np.add.reduceat(changed, offs[:-1]) == 1).all()            # one row per head took the new token
+        assert (cache.pos[torch.from_numpy(changed).cuda()] == wl.N + t).all()
+        gone = ev.cpu().numpy()
+        for u in range(wl.units):
+            assert gone[u] in pos_before[offs[u]:offs[u + 1]].cpu().numpy()
+            assert gone[u] not in cache.pos[offs[u]:offs[u + 1]].cpu().numpy()
