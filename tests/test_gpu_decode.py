@@ -223,3 +223,18 @@ def test_decode_cache_wrapper_runs_prefill_then_decode():
         for u in range(wl.units):
             assert gone[u] in pos_before[offs[u]:offs[u + 1]].cpu().numpy()
             assert gone[u] not in cache.pos[offs[u]:offs[u + 1]].cpu().numpy()
+
+
+def test_decode_many_small_caches():
+    """Many heads with tiny, uneven caches (1 to 40 rows), G = 2, fp32 and bf16: chunk and warp edges of every kernel."""
+    from paper_2410_03090_b200 import binding as ub
+    rng = np.random.default_rng(5)
+    for dtype in ("bf16", "fp32"):
+        B, L, H, Hq = 3, 4, 8, 16
+        units = B * L * H
+        caps = rng.integers(1, 41, size=units)
+        lens = np.minimum(caps, rng.integers(0, 41, size=units))
+        ctx = ub.Context(ub.make_shape(B, L, H, Hq, 512, 128, 8, dtype))
+        st = State(B, L, H, Hq, dtype, caps, lens, seed=23, start_pos=400)
+        for _ in range(3):
+            _step_and_check(ub, ctx, st, 40, protect=2)

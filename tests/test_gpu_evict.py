@@ -45,6 +45,9 @@ def _case(B, L, H, Hq, N, D, dtype, n_keep, layer, seed):
     (1, 2, 2, 16, 2049, 4096, "bf16", 512),      # G = 8, model-width rows of 8 KB
     (3, 1, 1, 16, 130, 64, "bf16", 1),           # G = 16; only the last position survives
     (1, 1, 8, 8, 513, 256, "bf16", 513),         # keep everything
+    (2, 1, 2, 4, 2, 8, "bf16", 1),               # two positions, 16-byte hidden rows
+    (1, 1, 1, 2, 33, 24, "fp32", 32),            # one past a warp of positions, drop exactly one
+    (5, 2, 4, 8, 1025, 72, "bf16", 7),           # one past a chunk, odd row width (144 bytes)
 ])
 def test_evict_hidden_parity(B, L, H, Hq, N, D, dtype, n_keep):
     idx = _case(B, L, H, Hq, N, D, dtype, n_keep, layer=L - 1, seed=N)
