@@ -45,6 +45,10 @@ def _check(ub, X, k, center, norm):
     (100, 256, 8, 32, 1, 1),        # token-space matrix padded from 100 to 128, whole-trace normalisation
     (1000, 4096, 50, 64, 1, 0),     # hidden-state width, short prompt
     (60, 512, 5, 64, 1, 0),         # k_trunc beyond the number of tokens: the missing eigenvalues are zero
+    (2, 128, 1, 8, 1, 0),           # two tokens: one non-zero eigenvalue after centring
+    (128, 128, 9, 32, 1, 0),        # square: the feature-space path at its smallest size
+    (129, 192, 9, 32, 0, 1),        # one token past a 64-token stage, token-space, uncentred, whole trace
+    (64, 4096, 4, 16, 1, 0),        # a single stage of tokens against the widest matrix
 ])
 def test_entropy_wide_parity(N, D, rank, k, center, norm):
     from paper_2410_03090_b200 import binding as ub
