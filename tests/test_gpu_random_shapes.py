@@ -12,26 +12,27 @@ from paper_2410_03090_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def _shape(rng, it):
+def _shape(rng, it, dtype="bf16"):
     H = rng.choice([1, 2, 4, 8])
     w = rng.choice([8, 16, 32, 64])
     G = min(rng.choice([1, 2, 4, 8]), 512 // w)
-    N = max(rng.choice([w + 9, 129, 257, 1000, 1537, 4097, 6000, 9001]), w + 9)
+    lengths = [w + 9, 129, 257, 1000, 1537, 4097, 6000, 9001] if dtype == "bf16" else [w + 9, 129, 257, 700, 1537]
+    N = max(rng.choice(lengths), w + 9)
     L, B = rng.choice([1, 2, 3]), rng.choice([1, 2])
     P = N - w
     avg = rng.randint(w + 1, max(w + 1, min(N - 1, w + P // 2)))
     M = rng.choice([m for m in (1, 2, 4, 8) if m <= H])
     n_max = min(N, max(avg, min(2 * avg - w, int(round(5 * avg / 3)))))
     return replace(synth.WORKLOADS["c2"], name=f"rnd{it}", B=B, L=L, H=H, Hq=H * G, N=N, w=w, avg_budget=avg, M=M,
-                   n_max=n_max, seed=1000 + it)
+                   n_max=n_max, seed=1000 + it, dtype=dtype)
 
 
-@pytest.mark.parametrize("seed", [1, 7])
-def test_random_shapes(seed):
+@pytest.mark.parametrize("seed,dtype,count", [(1, "bf16", 12), (7, "bf16", 12), (3, "fp32", 8)])
+def test_random_shapes(seed, dtype, count):
     from paper_2410_03090_b200.compress import CompressionPass
     rng = random.Random(seed)
-    for it in range(12):
-        wl = _shape(rng, it)
+    for it in range(count):
+        wl = _shape(rng, it, dtype)
         K, V, Qw = synth.generate(wl, "cuda")
         cp = CompressionPass(wl, "cuda")
         out = cp.run(K, V, Qw)
