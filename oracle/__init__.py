@@ -33,6 +33,8 @@ _lib.oracle_budgets.argtypes = [_dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int
 _lib.oracle_budgets.restype = C.c_int
 _lib.oracle_window_scores.argtypes = [_dp, _dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _dp]
 _lib.oracle_window_scores.restype = None
+_lib.oracle_window_lse.argtypes = [_dp, _dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _dp]
+_lib.oracle_window_lse.restype = None
 _lib.oracle_last_token_scores.argtypes = [_dp, _dp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_double, _dp]
 _lib.oracle_last_token_scores.restype = None
 _lib.oracle_decode_probs.argtypes = [_dp, _dp, _dp, C.c_int, C.c_int, C.c_int, C.c_double, _dp]
@@ -136,6 +138,18 @@ def window_scores(Q, K, scale: float | None = None) -> np.ndarray:
     raw = np.empty(N - w, dtype=np.float64)
     _lib.oracle_window_scores(_p(Q, _dp), _p(K, _dp), N, d, w, G, float(scale), _p(raw, _dp))
     return raw
+
+
+def window_lse(Q, K, scale: float | None = None) -> np.ndarray:
+    """Natural-log sum of exponentials of every window row's scaled, causally visible logits: [G, w]."""
+    Q, K = _f64(Q), _f64(K)
+    G, w, d = Q.shape
+    N = K.shape[0]
+    if scale is None:
+        scale = 1.0 / np.sqrt(float(d))
+    lse = np.empty((G, w), dtype=np.float64)
+    _lib.oracle_window_lse(_p(Q, _dp), _p(K, _dp), N, d, w, G, float(scale), _p(lse, _dp))
+    return lse
 
 
 def pool(raw, pool_kernel: int = 7, pool_mode: int = 0) -> np.ndarray:

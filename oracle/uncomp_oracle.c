@@ -14,7 +14,7 @@
  *   budgets               Section 3.3.3 ("Head-Group Compression", N_{i,g+1} = N_{i,g} - dn_g) and
  *                         Section 3.3.2 (layer-group partition: Delta c_i, C, N_{i+1} = N_i + dn)
  *   window scores         Section 3.3.3, "Dynamic KV Cache Eviction": attention of the last l query
- *                         positions summed per key position
+ *                         positions summed per key position; the log-sum-exp of each of those rows
  *   selection             same paragraph: keep the highest-scored tokens within the head's budget; the
  *                         recent (window) tokens are part of the budget (Section 4, recent/historical split)
  *   hidden-state eviction Section 3.3.2, "Hidden State Eviction": tokens kept for the next layer group by
@@ -320,6 +320,37 @@ void oracle_window_scores(const double *Q, const double *K, int N, int d, int w,
             double denom = 0.0;
             for (int j = 0; j <= last; ++j) denom += exp(s[j] - mx);
             for (int j = 0; j < P; ++j) raw[j] += exp(s[j] - mx) / denom;
+        }
+    }
+    free(s);
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Log-sum-exp of every window row (the row normaliser of the softmax above, Section 3.3.3): for query
+ * head g and window row i, lse[g * w + i] = ln sum_{j <= N - w + i} exp(scale * (q . k_j)), natural
+ * logarithm, over the same causally visible keys as oracle_window_scores.  It is what a prefill
+ * attention kernel keeps per row; with it, softmax(s)[j] = exp(s[j] - lse).  lse has G * w entries.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_window_lse(const double *Q, const double *K, int N, int d, int w, int G, double scale,
+                       double *lse)
+{
+    const int P = N - w;
+    double *s = (double *)malloc((size_t)N * sizeof(double));
+    for (int g = 0; g < G; ++g) {
+        for (int i = 0; i < w; ++i) {
+            const double *q = Q + ((size_t)g * w + i) * d;
+            const int last = P + i; /* inclusive */
+            double mx = -INFINITY;
+            for (int j = 0; j <= last; ++j) {
+                double acc = 0.0;
+                const double *k = K + (size_t)j * d;
+                for (int a = 0; a < d; ++a) acc += q[a] * k[a];
+                s[j] = scale * acc;
+                if (s[j] > mx) mx = s[j];
+            }
+            double denom = 0.0;
+            for (int j = 0; j <= last; ++j) denom += exp(s[j] - mx);
+            lse[(size_t)g * w + i] = mx + log(denom);
         }
     }
     free(s);

@@ -35,6 +35,36 @@ def test_scores_brute_force(N, w, G, d):
     np.testing.assert_allclose(oracle.window_scores(Q, K), _brute_scores(Q, K, scale), rtol=1e-12, atol=1e-15)
 
 
+@pytest.mark.parametrize("N,w,G,d", [(24, 4, 2, 8), (40, 7, 3, 16), (9, 1, 1, 4)])
+def test_window_lse_against_library_logsumexp_and_the_scores(N, w, G, d):
+    # pinned three ways: scipy's logsumexp of a numpy matrix product on every row's visible keys; the closed form
+    # for equal keys; and the identity softmax(s)[j] = exp(s[j] - lse), which must rebuild the window scores
+    from scipy.special import logsumexp
+    Q = RNG.normal(size=(G, w, d)) * 3.0
+    K = RNG.normal(size=(N, d))
+    scale = 0.37
+    P = N - w
+    lse = oracle.window_lse(Q, K, scale)
+    assert lse.shape == (G, w)
+    rebuilt = np.zeros(P)
+    for g in range(G):
+        for i in range(w):
+            lg = scale * (K[:P + i + 1] @ Q[g, i])
+            assert abs(lse[g, i] - logsumexp(lg)) < 1e-12 * max(1.0, abs(lse[g, i]))
+            rebuilt += np.exp(lg[:P] - lse[g, i])
+    np.testing.assert_allclose(rebuilt, oracle.window_scores(Q, K, scale), rtol=1e-12, atol=1e-300)
+    Ke = np.tile(K[:1], (N, 1))
+    lse_e = oracle.window_lse(Q, Ke, scale)
+    for g in range(G):
+        for i in range(w):
+            assert abs(lse_e[g, i] - (scale * float(Ke[0] @ Q[g, i]) + math.log(P + i + 1))) < 1e-12
+    # a key the row cannot see must not enter: changing the last key only moves the last row's value
+    K2 = K.copy()
+    K2[N - 1] += 5.0
+    d_lse = oracle.window_lse(Q, K2, scale) - lse
+    assert not np.any(d_lse[:, :w - 1]) and np.abs(d_lse[:, w - 1]).min() > 0.0
+
+
 def test_scores_equal_keys_closed_form():
     # all keys equal => every visible key gets 1/(number visible); raw[j] = G * sum_i 1/(N - w + i + 1)
     N, w, G, d = 40, 6, 3, 8
