@@ -70,7 +70,8 @@ enum {
 enum {
     UNCOMP_STATUS_NOT_CONVERGED = 1u, /* eigenvalue multi-section hit max_iters before its tolerance */
     UNCOMP_STATUS_TIMEOUT = 2u,       /* a bounded device-side wait expired */
-    UNCOMP_STATUS_BOUNDS = 4u         /* an index or budget check failed; the value was clamped / skipped */
+    UNCOMP_STATUS_BOUNDS = 4u,        /* an index, offset or budget check failed; the value was clamped / skipped */
+    UNCOMP_STATUS_NONFINITE = 8u      /* a caller-supplied log-sum-exp was NaN or infinite; its row was left out */
 };
 
 /* Bytes of device workspace a context of this shape needs.  Pure host function.  0 on a bad shape. */
@@ -93,18 +94,22 @@ void uncomp_destroy(uncomp_ctx *ctx);
  *   p_i = lambda_i / sum_{j<=k} lambda_j  (norm = 0)   or   lambda_i / trace(C)  (norm = 1)
  *   H_k = - sum_{i<=k} p_i ln p_i ,  erank_k = exp(H_k),   k = min(k_trunc, d)
  *
- * bf16 input: Gram matrix on the tensor cores with fp32 accumulation; fp32 input: fp64 accumulation.
- * The eigenvalues are computed in fp64 (Householder tridiagonalisation in shared memory, Sturm-count
- * multi-section for the k largest).  max_iters bounds the multi-section rounds (0 = default 14); a
- * unit that has not reached 1e-13 of its spectral radius by then sets UNCOMP_STATUS_NOT_CONVERGED
- * and still writes its current estimate.
+ * bf16 input: Gram matrix on the tensor cores with fp32 accumulation, chunk partials added in fp64, then
+ * an fp32 Householder tridiagonalisation held in registers and a Sturm-count multi-section for the k
+ * largest eigenvalues (bracketed to 2e-8 of the spectral radius; the fp32 reduction is good to about
+ * 1e-7).  fp32 input: Gram matrix and eigenvalues in fp64 throughout (Householder in shared memory,
+ * brackets to 1e-13 of the spectral radius).  max_iters bounds the multi-section rounds (0 = the default
+ * of the path, 10 or 14); a unit that has not reached its tolerance by then sets
+ * UNCOMP_STATUS_NOT_CONVERGED and still writes its current estimate.
  *
  * Fusion with the scorer: the window scorer (uncomp_score_select) also sweeps over K and needs, before
  * anything else, the softmax statistics of its window rows.  If d_Qw is given (bf16 keys only; ignored
  * otherwise), those statistics are produced in the same sweep that forms the Gram matrices -- one read of
  * K instead of two -- and are kept in the workspace.  The next uncomp_score_select call on this context
- * with the same d_K, strides, d_Qw and scale then skips its statistics pass.  The caller must not change
- * K or Qw in between.  d_Qw = NULL runs the entropy stage on its own.
+ * skips its statistics pass if it sets reuse_stats = 1 and passes the same d_K, strides, d_Qw and scale;
+ * by setting the flag the caller vouches that K and Qw have not changed in between (the library compares
+ * pointers, it cannot see contents).  Any uncomp_score_select call consumes the statistics.
+ * d_Qw = NULL runs the entropy stage on its own.
  *
  * d_K        in   [B, L, H, N, d] with strides sK, storage dtype of the shape
  * d_Qw       in   [B, L, Hq, w, d] window queries as for uncomp_score_select, or NULL
@@ -142,16 +147,20 @@ int uncomp_gram(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, double *d_g
  * The call itself allocates nothing, on the device or through any library.
  *
  * Limits and rules
- *   - (units) x (token chunks per unit) partials must fit the array: at most 64 partials for bf16 keys,
- *     32 for fp32 keys (e.g. 8 heads x 32768 tokens in bf16 is 8 x 8 = 64).  Larger shapes are refused
- *     with UNCOMP_E_LIMIT and nothing is launched.
+ *   - The array holds 64 chunk partials for bf16 keys and 32 for fp32 keys, and every unit needs at least
+ *     one: at most 64 (32) units per call, any number of tokens.  More units are refused with
+ *     UNCOMP_E_LIMIT and nothing is launched.  When units x (token chunks uncomp_gram would use) exceeds
+ *     the array, the call takes fewer, longer chunks (e.g. one layer of 8 heads x 32768 tokens in bf16 runs
+ *     as 8 x 8 chunks of 4096 tokens instead of 8 x 32).  A chunk is accumulated in fp32 on the tensor
+ *     cores, so longer chunks round more: about 1e-5 of the largest entry at 4096 tokens per chunk, against
+ *     2e-6 at uncomp_gram's 1024; with the same chunking the two entry points agree bit for bit.
  *   - The first call on a device looks up the array's device address (the device must be current).  Make
  *     that first call outside any stream capture.
  *   - All calls share the one array and it keeps the previous call's contents; this call overwrites the
  *     part it reads and clears its status word itself.  Two calls whose GPU work overlaps (different
  *     streams, or threads) race on it: serialise them.
  *   - Device-side conditions (a bounded wait that expired) are not reported by this entry point.
- * Arguments as for uncomp_gram, with the shape passed directly; the result is identical to uncomp_gram's. */
+ * Arguments as for uncomp_gram, with the shape passed directly. */
 int uncomp_gram_static(const uncomp_shape *shape, const void *d_K, uncomp_strides sK, double *d_gram, void *stream);
 size_t uncomp_gram_static_max_bytes(void);
 
@@ -206,11 +215,27 @@ int uncomp_assign_budgets(uncomp_ctx *ctx, const float *d_erank, const uncomp_bu
  *              clipped to the prefix.
  * The budget[u] - w prefix positions with the largest score (ties: lower position) are written in
  * ascending order to d_indices[offsets[u] ...], followed by the window positions N-w .. N-1.
- * A budget outside [w, N] is clamped and sets UNCOMP_STATUS_BOUNDS.
+ *
+ * Softmax needs every row's normaliser before any column can be summed, so the window logits are formed
+ * twice (a statistics sweep over K, then the column sums) unless the normalisers are already known:
+ *   - reuse_stats = 1: a preceding uncomp_entropy call with d_Qw left them in the workspace (see there);
+ *   - d_lse given: the caller supplies them.  A prefill attention kernel that has just processed the same
+ *     window rows owns, per row, lse = ln sum_{j' visible} exp(s_{q,i}[j']) (natural logarithm, of the
+ *     SCALED logits, over all causally visible keys, prefix and window alike).  Then
+ *     softmax(s)[j] = exp(s[j] - lse) and one sweep over K suffices.  The values are trusted: an lse that
+ *     does not belong to these queries and keys gives scores that are wrong by the same factor.  A NaN or
+ *     infinite entry sets UNCOMP_STATUS_NONFINITE and its row contributes nothing.
+ *
+ * Every slab offsets[u] .. offsets[u+1] is filled completely and nothing is written outside it: a budget
+ * that differs from the slab length or lies outside [w, N], or offsets that are not ascending inside
+ * [0, offsets[units]], set UNCOMP_STATUS_BOUNDS; the unit then keeps as many top positions as the slab and
+ * the budget allow, the window positions as far as they fit, and fills what remains with position N - 1
+ * (a unit whose offsets are unusable writes nothing).
  *
  * d_Qw       in   [B, L, Hq, w, d] contiguous, storage dtype; query head q belongs to KV head q / G
  * d_K        in   as in uncomp_entropy
- * d_budgets  in   [B, L, H] int32, each in [w, N]
+ * d_lse      in   [B, L, Hq, w] float, or NULL
+ * d_budgets  in   [B, L, H] int32, each in [w, N] and equal to offsets[u+1] - offsets[u]
  * d_offsets  in   [B*L*H + 1] int64
  * d_scores   out  [B, L, H, N - w] float, the pooled scores; may be NULL (workspace is used then)
  * d_indices  out  [offsets[units]] int32
@@ -219,9 +244,12 @@ typedef struct {
     int32_t pool_kernel; /* odd, 1 = no pooling, at most 63 */
     int32_t pool_mode;   /* 0 = max, 1 = mean */
     float scale;         /* 0 means 1 / sqrt(d) */
+    int32_t reuse_stats; /* 1 = take the row statistics the preceding uncomp_entropy (with d_Qw) left for these
+                            d_K, strides, d_Qw and scale; when there are none (another tensor, fp32 keys) the
+                            statistics sweep runs as with 0.  0 = never reuse.  Ignored when d_lse is given. */
 } uncomp_score_params;
 
-int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, uncomp_strides sK,
+int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, uncomp_strides sK, const float *d_lse,
                         const int32_t *d_budgets, const int64_t *d_offsets, const uncomp_score_params *params,
                         float *d_scores, int32_t *d_indices, void *stream);
 
@@ -229,7 +257,8 @@ int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, unco
  * uncomp_compact -- the per-head ragged cache of Section 3.3.3 ("each head maintains its context
  * window"); keys and values share one selection (caption of the paper's main table).
  *   Kc[offsets[u] + t, :] = K[unit u, indices[offsets[u] + t], :]   for t < offsets[u+1] - offsets[u]
- * and the same for V.  Rows are copied bit for bit.
+ * and the same for V.  Rows are copied bit for bit.  An index outside [0, N) is replaced by the nearest
+ * valid position and sets UNCOMP_STATUS_BOUNDS (no address outside the unit's rows is ever formed).
  *
  * d_K, d_V    in   [B, L, H, N, d] with strides sK, sV
  * d_indices   in   [offsets[units]] int32

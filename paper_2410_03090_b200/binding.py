@@ -18,7 +18,7 @@ UNCOMP_BF16, UNCOMP_FP32 = 0, 1
 UNCOMP_OK = 0
 UNCOMP_E_NULL, UNCOMP_E_SHAPE, UNCOMP_E_ALIGN, UNCOMP_E_WORKSPACE = -1, -2, -3, -4
 UNCOMP_E_PARAM, UNCOMP_E_CUDA, UNCOMP_E_LIMIT = -5, -6, -7
-UNCOMP_STATUS_NOT_CONVERGED, UNCOMP_STATUS_TIMEOUT, UNCOMP_STATUS_BOUNDS = 1, 2, 4
+UNCOMP_STATUS_NOT_CONVERGED, UNCOMP_STATUS_TIMEOUT, UNCOMP_STATUS_BOUNDS, UNCOMP_STATUS_NONFINITE = 1, 2, 4, 8
 
 
 class uncomp_shape(C.Structure):
@@ -39,7 +39,8 @@ class uncomp_budget_params(C.Structure):
 
 
 class uncomp_score_params(C.Structure):
-    _fields_ = [("pool_kernel", C.c_int32), ("pool_mode", C.c_int32), ("scale", C.c_float)]
+    _fields_ = [("pool_kernel", C.c_int32), ("pool_mode", C.c_int32), ("scale", C.c_float),
+                ("reuse_stats", C.c_int32)]
 
 
 def _load() -> C.CDLL:
@@ -69,7 +70,7 @@ def _load() -> C.CDLL:
     lib.uncomp_assign_budgets.restype = C.c_int
     lib.uncomp_assign_budgets.argtypes = [vp, fp, C.POINTER(uncomp_budget_params), i32p, i64p, i32p, i32p, vp]
     lib.uncomp_score_select.restype = C.c_int
-    lib.uncomp_score_select.argtypes = [vp, vp, vp, uncomp_strides, i32p, i64p, C.POINTER(uncomp_score_params),
+    lib.uncomp_score_select.argtypes = [vp, vp, vp, uncomp_strides, fp, i32p, i64p, C.POINTER(uncomp_score_params),
                                         fp, i32p, vp]
     lib.uncomp_compact.restype = C.c_int
     lib.uncomp_compact.argtypes = [vp, vp, vp, uncomp_strides, uncomp_strides, i32p, i64p, vp, vp, vp]
@@ -227,12 +228,19 @@ def uncomp_assign_budgets(ctx: Context, erank: torch.Tensor, avg_budget: int, M:
 def uncomp_score_select(ctx: Context, Qw: torch.Tensor, K: torch.Tensor, budgets: torch.Tensor,
                         offsets: torch.Tensor, total_rows: int, pool_kernel: int = 7, pool_mode: int = 0,
                         scale: float = 0.0, scores: Optional[torch.Tensor] = None,
-                        indices: Optional[torch.Tensor] = None, stream=None):
+                        indices: Optional[torch.Tensor] = None, stream=None, lse: Optional[torch.Tensor] = None,
+                        reuse_stats: bool = False):
+    """lse [B, L, Hq, w] float32 (natural-log sum of exponentials of every window row's scaled logits): the
+    caller's softmax normalisers, one sweep over K instead of two.  reuse_stats: take the statistics a preceding
+    uncomp_entropy(..., Qw=Qw) left in the workspace."""
     if indices is None:
         indices = torch.empty(total_rows, dtype=torch.int32, device=K.device)
-    p = uncomp_score_params(pool_kernel, pool_mode, scale)
-    _check(lib.uncomp_score_select(ctx.handle, _ptr(Qw), _ptr(K), strides_of(K), _ptr(budgets), _ptr(offsets),
-                                   C.byref(p), _ptr(scores), _ptr(indices), _stream(stream)), "uncomp_score_select")
+    if lse is not None and (lse.dtype != torch.float32 or not lse.is_contiguous()):
+        raise ValueError("lse must be a contiguous float32 tensor [B, L, Hq, w]")
+    p = uncomp_score_params(pool_kernel, pool_mode, scale, int(reuse_stats))
+    _check(lib.uncomp_score_select(ctx.handle, _ptr(Qw), _ptr(K), strides_of(K), _ptr(lse), _ptr(budgets),
+                                   _ptr(offsets), C.byref(p), _ptr(scores), _ptr(indices), _stream(stream)),
+           "uncomp_score_select")
     return indices
 
 

@@ -49,14 +49,18 @@ class CompressionPass:
         )
 
     def score(self, K: torch.Tensor, Qw: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
-              eps: float = 0.0, dn: int = 0, n_last: int = 0, scope: int = 0) -> PassOutput:
-        """Everything that needs only the keys and the window queries: entropy, budgets, scores, kept positions."""
+              eps: float = 0.0, dn: int = 0, n_last: int = 0, scope: int = 0,
+              lse: Optional[torch.Tensor] = None) -> PassOutput:
+        """Everything that needs only the keys and the window queries: entropy, budgets, scores, kept positions.
+        With `lse` (the caller's log-sum-exp of every window row, [B, L, Hq, w] float32) the scorer makes one sweep
+        over K and the entropy call runs the Gram stage on its own."""
         wl, o, ctx = self.wl, self.out, self.ctx
-        ub.uncomp_entropy(ctx, K, wl.k_trunc, 1, 0, 0, o.entropy, o.erank, None, stream, Qw=Qw if self.fused else None)
+        fuse = self.fused and lse is None and wl.dtype == "bf16"
+        ub.uncomp_entropy(ctx, K, wl.k_trunc, 1, 0, 0, o.entropy, o.erank, None, stream, Qw=Qw if fuse else None)
         ub.uncomp_assign_budgets(ctx, o.erank, wl.avg_budget, wl.M, wl.n_max, scope, eps, dn, n_last,
                                  o.budgets, o.offsets, o.layer_group, o.layer_ctx, stream)
         ub.uncomp_score_select(ctx, Qw, K, o.budgets, o.offsets, wl.total_rows, wl.pool_kernel, wl.pool_mode, 0.0,
-                               o.scores, o.indices, stream)
+                               o.scores, o.indices, stream, lse=lse, reuse_stats=fuse)
         return o
 
     def compact(self, K: torch.Tensor, V: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> PassOutput:
@@ -66,8 +70,9 @@ class CompressionPass:
         return o
 
     def run(self, K: torch.Tensor, V: torch.Tensor, Qw: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
-            eps: float = 0.0, dn: int = 0, n_last: int = 0, scope: int = 0) -> PassOutput:
-        self.score(K, Qw, stream, eps, dn, n_last, scope)
+            eps: float = 0.0, dn: int = 0, n_last: int = 0, scope: int = 0,
+            lse: Optional[torch.Tensor] = None) -> PassOutput:
+        self.score(K, Qw, stream, eps, dn, n_last, scope, lse)
         return self.compact(K, V, stream)
 
     def status(self, stream=None) -> int:

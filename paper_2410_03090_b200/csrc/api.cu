@@ -4,7 +4,7 @@
 #include <new>
 #include <vector>
 
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace uncomp {
 
@@ -29,7 +29,9 @@ Plan make_plan(const uncomp_shape &s) {
     p.G = s.Hq / s.H;
     p.rows = p.G * s.w;
     p.prefix = s.N - s.w;
-    const int target_ctas = 592;   // four CTAs for each of the 148 SMs
+    // Four CTAs per SM of the target part.  The plan (and with it the workspace size) must not depend on the
+    // device that happens to be present: uncomp_workspace_bytes is a pure host function.
+    const int target_ctas = 4 * kTargetSms;
     {
         int want = (target_ctas + p.units - 1) / p.units;
         int most = (s.N + 1023) / 1024;
@@ -111,6 +113,7 @@ struct uncomp_ctx {
     const void *stats_K, *stats_Qw;
     uncomp_strides stats_sK;
     float stats_scale;
+    TmapCache tmaps;  // tensor maps of the last key / query tensors the scorer saw
 };
 
 static int cuda_fail(uncomp_ctx *ctx, cudaError_t e) {
@@ -169,6 +172,7 @@ int uncomp_create(uncomp_ctx **out, const uncomp_shape *shape, void *d_workspace
     ctx->prof = nullptr;
     ctx->force_simt = 0;
     ctx->stats_valid = 0;
+    ctx->tmaps.k_valid = ctx->tmaps.q_valid = false;
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) e = cudaMemset(ctx->ws + p.off_status, 0, 256);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -189,7 +193,11 @@ void uncomp_destroy(uncomp_ctx *ctx) {
 
 int uncomp_set_option(uncomp_ctx *ctx, int option, int value) {
     if (!ctx) return UNCOMP_E_NULL;
-    if (option == UNCOMP_OPT_CUDA_CORES) { ctx->force_simt = value != 0; return UNCOMP_OK; }
+    if (option == UNCOMP_OPT_CUDA_CORES) {
+        ctx->force_simt = value != 0;
+        ctx->stats_valid = 0;      // the two kernel families keep their statistics in different formats
+        return UNCOMP_OK;
+    }
     return UNCOMP_E_PARAM;
 }
 
@@ -257,9 +265,9 @@ int uncomp_entropy(uncomp_ctx *ctx, const void *d_K, uncomp_strides sK, const un
     if (tensor_path && d_Qw) {
         // one sweep over K: Gram partials per scorer chunk and the scorer's row statistics
         const float sc = effective_scale(scale, p.shape.d);
-        e = launch_scores_tc(p, d_Qw, d_K, addr, sc, reinterpret_cast<float *>(ctx->ws + p.off_stats_part),
+        e = launch_scores_tc(p, d_Qw, d_K, addr, sc, nullptr, reinterpret_cast<float *>(ctx->ws + p.off_stats_part),
                              reinterpret_cast<float *>(ctx->ws + p.off_stats), nullptr,
-                             reinterpret_cast<float *>(partials), kScorePhaseStats, d_status, ctx->prof, st);
+                             reinterpret_cast<float *>(partials), kScorePhaseStats, d_status, &ctx->tmaps, ctx->prof, st);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
         parts = p.score_splits;
         ctx->stats_valid = 1;
@@ -324,18 +332,26 @@ int uncomp_assign_budgets(uncomp_ctx *ctx, const float *d_erank, const uncomp_bu
     return UNCOMP_OK;
 }
 
-int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, uncomp_strides sK,
+int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, uncomp_strides sK, const float *d_lse,
                         const int32_t *d_budgets, const int64_t *d_offsets, const uncomp_score_params *params,
                         float *d_scores, int32_t *d_indices, void *stream) {
     if (!ctx || !d_Qw || !d_K || !d_budgets || !d_offsets || !params || !d_indices) return UNCOMP_E_NULL;
     const Plan &p = ctx->plan;
     if (!aligned16(d_K) || !aligned16(d_Qw)) return UNCOMP_E_ALIGN;
+    if (d_lse && (reinterpret_cast<uintptr_t>(d_lse) & 3u)) return UNCOMP_E_ALIGN;
     int rc = check_strides(p.shape, sK);
     if (rc != UNCOMP_OK) return rc;
     if (params->pool_kernel < 1 || params->pool_kernel > 63 || (params->pool_kernel & 1) == 0 ||
-        (params->pool_mode != 0 && params->pool_mode != 1) || !(params->scale >= 0.f) || isinf(params->scale))
+        (params->pool_mode != 0 && params->pool_mode != 1) || !(params->scale >= 0.f) || isinf(params->scale) ||
+        (params->reuse_stats != 0 && params->reuse_stats != 1))
         return UNCOMP_E_PARAM;
     const float scale = effective_scale(params->scale, p.shape.d);
+    const bool tensor_path = p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt;
+    // row statistics: supplied by the caller (d_lse), left by a fused uncomp_entropy call (reuse_stats), or
+    // produced here by a statistics sweep of their own
+    const bool reuse = !d_lse && params->reuse_stats && tensor_path && ctx->stats_valid && ctx->stats_K == d_K &&
+                       ctx->stats_Qw == d_Qw && same_strides(ctx->stats_sK, sK) && ctx->stats_scale == scale;
+    ctx->stats_valid = 0;          // every path below overwrites the statistics region or consumes it
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint32_t *d_status = reinterpret_cast<uint32_t *>(ctx->ws + p.off_status);
     float *stats_part = reinterpret_cast<float *>(ctx->ws + p.off_stats_part);
@@ -344,15 +360,12 @@ int uncomp_score_select(uncomp_ctx *ctx, const void *d_Qw, const void *d_K, unco
     float *pooled = d_scores ? d_scores : reinterpret_cast<float *>(ctx->ws + p.off_pooled);
     const UnitAddr addr = make_addr(p.shape, sK);
     cudaError_t e;
-    if (p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt) {
-        // the statistics pass is skipped when a fused uncomp_entropy call left them for exactly these inputs
-        const bool reuse = ctx->stats_valid && ctx->stats_K == d_K && ctx->stats_Qw == d_Qw &&
-                           same_strides(ctx->stats_sK, sK) && ctx->stats_scale == scale;
-        ctx->stats_valid = 0;
-        const int phases = reuse ? kScorePhaseColsum : (kScorePhaseStats | kScorePhaseColsum);
-        e = launch_scores_tc(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, nullptr, phases, d_status, ctx->prof, st);
+    if (tensor_path) {
+        const int phases = (reuse || d_lse) ? kScorePhaseColsum : (kScorePhaseStats | kScorePhaseColsum);
+        e = launch_scores_tc(p, d_Qw, d_K, addr, scale, d_lse, stats_part, stats, raw, nullptr, phases, d_status,
+                             &ctx->tmaps, ctx->prof, st);
     } else {
-        e = launch_scores_simt(p, d_Qw, d_K, addr, scale, stats_part, stats, raw, ctx->prof, st);
+        e = launch_scores_simt(p, d_Qw, d_K, addr, scale, d_lse, stats_part, stats, raw, d_status, ctx->prof, st);
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     {
@@ -378,7 +391,7 @@ int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_str
     {
         ProfScope ps(ctx->prof, kSlotCompact, st);
         e = launch_compact(p, d_K, d_V, make_addr(p.shape, sK), make_addr(p.shape, sV), d_indices, d_offsets, d_Kc,
-                           d_Vc, st);
+                           d_Vc, reinterpret_cast<uint32_t *>(ctx->ws + p.off_status), st);
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;

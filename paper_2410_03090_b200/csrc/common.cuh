@@ -11,6 +11,7 @@ namespace uncomp {
 
 constexpr int kD = 128;          // head dimension supported by every kernel
 constexpr int kMaxRows = 512;    // G * w upper bound (window rows of all grouped query heads)
+constexpr int kTargetSms = 148;  // SM count of the part the grids are sized for (B200)
 
 // Carve-up of the caller's workspace, decided by the shape alone (see api.cu).
 struct Plan {
@@ -91,13 +92,21 @@ int check_budget_params(const uncomp_shape &s, const uncomp_budget_params &bp);
 cudaError_t launch_budgets(const Plan &p, const float *d_erank, const uncomp_budget_params &bp, int32_t *d_budgets,
                            int64_t *d_offsets, int32_t *d_layer_group, int32_t *d_layer_ctx, int32_t *d_rank,
                            int64_t *d_rem, cudaStream_t st);
+// d_lse != NULL: the caller's log-sum-exp per window row replaces the statistics pass and the merge
 cudaError_t launch_scores_simt(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
-                               float *d_stats_part, float *d_stats, float *d_raw, Profiler *prof, cudaStream_t st);
+                               const float *d_lse, float *d_stats_part, float *d_stats, float *d_raw,
+                               uint32_t *d_status, Profiler *prof, cudaStream_t st);
+// Caller-supplied ln-sum-exp [units, rows] -> the merged statistics the column-sum kernels read: m' = lse * log2(e)
+// per row (log2_domain, tensor-core kernels) or the pair (lse, 1) (CUDA-core kernels).  A non-finite entry raises
+// UNCOMP_STATUS_NONFINITE and becomes +inf, so that its row adds nothing.
+cudaError_t launch_lse_import(const Plan &p, const float *d_lse, float *d_stats, bool log2_domain, uint32_t *d_status,
+                              cudaStream_t st);
+struct TmapCache;
 // phases: kScorePhaseStats (pass A; with d_gram_part != NULL the Gram partials of every (unit, scorer chunk) are
-// produced in the same sweep) and / or kScorePhaseColsum (merge + pass B)
+// produced in the same sweep) and / or kScorePhaseColsum (merge, or the import of d_lse when given, + pass B)
 cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
-                             float *d_stats_part, float *d_stats, float *d_raw, float *d_gram_part, int phases,
-                             uint32_t *d_status, Profiler *prof, cudaStream_t st);
+                             const float *d_lse, float *d_stats_part, float *d_stats, float *d_raw, float *d_gram_part,
+                             int phases, uint32_t *d_status, TmapCache *cache, Profiler *prof, cudaStream_t st);
 cudaError_t launch_pool_select(const Plan &p, const float *d_raw, float *d_pooled, int pool_kernel, int pool_mode,
                                const int32_t *d_budgets, const int64_t *d_offsets, int32_t *d_indices,
                                uint32_t *d_status, cudaStream_t st);
@@ -126,6 +135,6 @@ cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const
                                 uint32_t *d_status, Profiler *prof, cudaStream_t st);
 cudaError_t launch_compact(const Plan &p, const void *dK, const void *dV, const UnitAddr &aK, const UnitAddr &aV,
                            const int32_t *d_indices, const int64_t *d_offsets, void *dKc, void *dVc,
-                           cudaStream_t st);
+                           uint32_t *d_status, cudaStream_t st);
 
 }  // namespace uncomp

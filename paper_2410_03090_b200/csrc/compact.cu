@@ -14,11 +14,12 @@ namespace uncomp {
 template <int ROW_BYTES>
 __global__ void __launch_bounds__(256) compact_kernel(const unsigned char *__restrict__ K,
                                                       const unsigned char *__restrict__ V, UnitAddr aK, UnitAddr aV,
-                                                      int units, int elem_bytes,
+                                                      int units, int N, int elem_bytes,
                                                       const int32_t *__restrict__ indices,
                                                       const int64_t *__restrict__ offsets,
                                                       unsigned char *__restrict__ Kc,
-                                                      unsigned char *__restrict__ Vc) {
+                                                      unsigned char *__restrict__ Vc,
+                                                      uint32_t *__restrict__ status) {
     constexpr int LANES_PER_ROW = ROW_BYTES / 16;          // 16 or 32
     constexpr int ROWS_PER_STEP = 32 / LANES_PER_ROW;      // 2 or 1
     const int lane = threadIdx.x & 31;
@@ -35,7 +36,11 @@ __global__ void __launch_bounds__(256) compact_kernel(const unsigned char *__res
                 const int mid = (lo + hi + 1) >> 1;
                 if (offsets[mid] <= t) lo = mid; else hi = mid - 1;
             }
-            const int64_t idx = indices[t];
+            int64_t idx = indices[t];
+            if (idx < 0 || idx >= N) {        // never form an address outside the unit's rows
+                atomicOr(status, (uint32_t)UNCOMP_STATUS_BOUNDS);
+                idx = idx < 0 ? 0 : N - 1;
+            }
             srcK = (aK.base(lo) + idx * aK.sN) * elem_bytes;
             srcV = (aV.base(lo) + idx * aV.sN) * elem_bytes;
         }
@@ -58,19 +63,19 @@ __global__ void __launch_bounds__(256) compact_kernel(const unsigned char *__res
 
 cudaError_t launch_compact(const Plan &p, const void *dK, const void *dV, const UnitAddr &aK, const UnitAddr &aV,
                            const int32_t *d_indices, const int64_t *d_offsets, void *dKc, void *dVc,
-                           cudaStream_t st) {
+                           uint32_t *d_status, cudaStream_t st) {
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int grid = sms * 8;
     if (p.shape.dtype == UNCOMP_FP32)
         compact_kernel<512><<<grid, 256, 0, st>>>((const unsigned char *)dK, (const unsigned char *)dV, aK, aV,
-                                                  p.units, 4, d_indices, d_offsets, (unsigned char *)dKc,
-                                                  (unsigned char *)dVc);
+                                                  p.units, p.shape.N, 4, d_indices, d_offsets, (unsigned char *)dKc,
+                                                  (unsigned char *)dVc, d_status);
     else
         compact_kernel<256><<<grid, 256, 0, st>>>((const unsigned char *)dK, (const unsigned char *)dV, aK, aV,
-                                                  p.units, 2, d_indices, d_offsets, (unsigned char *)dKc,
-                                                  (unsigned char *)dVc);
+                                                  p.units, p.shape.N, 2, d_indices, d_offsets, (unsigned char *)dKc,
+                                                  (unsigned char *)dVc, d_status);
     return cudaGetLastError();
 }
 

@@ -58,10 +58,17 @@ extern "C" int uncomp_gram_static(const uncomp_shape *shape, const void *d_K, un
         if ((st[i] * eb) % 16 != 0) return UNCOMP_E_ALIGN;
     }
     if (sK.sN < shape->d) return UNCOMP_E_SHAPE;
-    const Plan p = make_plan(*shape);
+    Plan p = make_plan(*shape);
     const size_t acc = shape->dtype == UNCOMP_FP32 ? sizeof(double) : sizeof(float);
-    const size_t need = (size_t)p.units * p.gram_splits * kPartialLen * acc;
-    if (need > kStaticScratchBytes) return UNCOMP_E_LIMIT;      // more (unit, chunk) partials than the array holds
+    const size_t slots = kStaticScratchBytes / (kPartialLen * acc);      // partials the array holds: 64 or 32
+    if ((size_t)p.units > slots) return UNCOMP_E_LIMIT;                  // not even one partial per unit
+    if ((size_t)p.units * p.gram_splits > slots) {
+        // fewer, longer token chunks than the workspace entry point would use, so that the partials fit
+        const int splits = (int)(slots / p.units);
+        const int chunk = ((shape->N + splits - 1) / splits + 127) / 128 * 128;
+        p.gram_chunk = chunk;
+        p.gram_splits = (shape->N + chunk - 1) / chunk;
+    }
 
     void *scratch = nullptr;
     if (scratch_address(&scratch) != cudaSuccess) return UNCOMP_E_CUDA;

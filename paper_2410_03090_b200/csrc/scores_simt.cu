@@ -171,10 +171,37 @@ __global__ void __launch_bounds__(256) score_colsum_simt_kernel(const T *__restr
     }
 }
 
+// one thread per (unit, row): the caller's natural-log sum of exponentials in place of pass A and the merge
+__global__ void lse_import_kernel(const float *__restrict__ lse, int units, int rows, int log2_domain,
+                                  float *__restrict__ stats, uint32_t *__restrict__ status) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= units * rows) return;
+    const int u = idx / rows, r = idx % rows;
+    float v = lse[idx];
+    if (!isfinite(v)) {
+        atomicOr(status, (uint32_t)UNCOMP_STATUS_NONFINITE);
+        v = INFINITY;                        // exp(s - inf) = 0: the row drops out of every column sum
+    }
+    if (log2_domain) {
+        stats[(size_t)u * kMaxRows + r] = v * 1.4426950408889634f;
+    } else {
+        stats[((size_t)u * kMaxRows + r) * 2] = v;
+        stats[((size_t)u * kMaxRows + r) * 2 + 1] = 1.f;
+    }
+}
+
+cudaError_t launch_lse_import(const Plan &p, const float *d_lse, float *d_stats, bool log2_domain, uint32_t *d_status,
+                              cudaStream_t st) {
+    const int total = p.units * p.rows;
+    lse_import_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_lse, p.units, p.rows, log2_domain ? 1 : 0, d_stats,
+                                                           d_status);
+    return cudaGetLastError();
+}
+
 template <typename T>
 static cudaError_t launch_scores_simt_t(const Plan &p, const T *dQw, const T *dK, const UnitAddr &addr, float scale,
-                                        float *d_stats_part, float *d_stats, float *d_raw, Profiler *prof,
-                                        cudaStream_t st) {
+                                        const float *d_lse, float *d_stats_part, float *d_stats, float *d_raw,
+                                        uint32_t *d_status, Profiler *prof, cudaStream_t st) {
     const size_t smemA = 2 * kSB * kKPad * sizeof(float);
     const size_t smemB = smemA + 16 * kSB * sizeof(float);
     cudaError_t e = cudaFuncSetAttribute(score_stats_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -182,15 +209,19 @@ static cudaError_t launch_scores_simt_t(const Plan &p, const T *dQw, const T *dK
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(score_colsum_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smemB);
     if (e != cudaSuccess) return e;
-    const int row_blocks = (p.rows + kSB - 1) / kSB;
-    dim3 gA(p.score_splits, row_blocks, p.units);
-    {
-        ProfScope ps(prof, kSlotScoreStats, st);
-        score_stats_simt_kernel<T><<<gA, 256, smemA, st>>>(dQw, dK, addr, p.shape.N, p.shape.w, p.G, p.score_chunk,
-                                                           p.score_splits, scale, d_stats_part);
-    }
-    const int total = p.units * p.rows;
-    {
+    if (d_lse) {
+        ProfScope ps(prof, kSlotStatsMerge, st);
+        e = launch_lse_import(p, d_lse, d_stats, false, d_status, st);
+        if (e != cudaSuccess) return e;
+    } else {
+        const int row_blocks = (p.rows + kSB - 1) / kSB;
+        dim3 gA(p.score_splits, row_blocks, p.units);
+        {
+            ProfScope ps(prof, kSlotScoreStats, st);
+            score_stats_simt_kernel<T><<<gA, 256, smemA, st>>>(dQw, dK, addr, p.shape.N, p.shape.w, p.G, p.score_chunk,
+                                                               p.score_splits, scale, d_stats_part);
+        }
+        const int total = p.units * p.rows;
         ProfScope ps(prof, kSlotStatsMerge, st);
         score_stats_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows, p.score_splits,
                                                                       d_stats);
@@ -205,12 +236,13 @@ static cudaError_t launch_scores_simt_t(const Plan &p, const T *dQw, const T *dK
 }
 
 cudaError_t launch_scores_simt(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
-                               float *d_stats_part, float *d_stats, float *d_raw, Profiler *prof, cudaStream_t st) {
+                               const float *d_lse, float *d_stats_part, float *d_stats, float *d_raw,
+                               uint32_t *d_status, Profiler *prof, cudaStream_t st) {
     if (p.shape.dtype == UNCOMP_FP32)
-        return launch_scores_simt_t<float>(p, (const float *)dQw, (const float *)dK, addr, scale, d_stats_part,
-                                           d_stats, d_raw, prof, st);
+        return launch_scores_simt_t<float>(p, (const float *)dQw, (const float *)dK, addr, scale, d_lse, d_stats_part,
+                                           d_stats, d_raw, d_status, prof, st);
     return launch_scores_simt_t<__nv_bfloat16>(p, (const __nv_bfloat16 *)dQw, (const __nv_bfloat16 *)dK, addr, scale,
-                                               d_stats_part, d_stats, d_raw, prof, st);
+                                               d_lse, d_stats_part, d_stats, d_raw, d_status, prof, st);
 }
 
 }  // namespace uncomp

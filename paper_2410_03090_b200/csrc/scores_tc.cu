@@ -413,15 +413,30 @@ __global__ void score_tc_merge_kernel(const float *__restrict__ stats_part, int 
     mprime[(size_t)u * kMaxRows + r] = m + log2f(l);
 }
 
+// cudaFuncSetAttribute is sticky per function and device: done once per device and instantiation
 template <int MB>
-static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, const CUtensorMap &tk, float c_log2,
-                                       float *d_stats_part, float *d_mprime, float *d_raw, float *d_gram_part,
-                                       int phases, uint32_t *d_status, Profiler *prof, cudaStream_t st) {
-    const uncomp_shape &s = p.shape;
+static cudaError_t raise_smem_limit_once() {
+    static bool done[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
     const int smem = score_smem(MB);
-    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<MB, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    e = cudaFuncSetAttribute(score_tc_kernel<MB, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(score_tc_kernel<MB, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(score_tc_kernel<MB, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+    return e;
+}
+
+template <int MB>
+static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, const CUtensorMap &tk, float c_log2,
+                                       const float *d_lse, float *d_stats_part, float *d_mprime, float *d_raw,
+                                       float *d_gram_part, int phases, uint32_t *d_status, Profiler *prof,
+                                       cudaStream_t st) {
+    const uncomp_shape &s = p.shape;
+    const int smem = score_smem(MB);
+    cudaError_t e = raise_smem_limit_once<MB>();
     if (e != cudaSuccess) return e;
     if (phases & kScorePhaseStats) {
         ProfScope ps(prof, d_gram_part ? kSlotGramStats : kSlotScoreStats, st);
@@ -438,9 +453,14 @@ static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, con
     if (phases & kScorePhaseColsum) {
         {
             ProfScope ps(prof, kSlotStatsMerge, st);
-            const int total = p.units * p.rows;
-            score_tc_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows, p.score_splits,
-                                                                       d_mprime);
+            if (d_lse) {
+                e = launch_lse_import(p, d_lse, d_mprime, true, d_status, st);
+                if (e != cudaSuccess) return e;
+            } else {
+                const int total = p.units * p.rows;
+                score_tc_merge_kernel<<<(total + 255) / 256, 256, 0, st>>>(d_stats_part, p.units, p.rows,
+                                                                           p.score_splits, d_mprime);
+            }
         }
         ProfScope ps(prof, kSlotScoreColsum, st);
         const int splitsB = (p.prefix + p.score_chunk - 1) / p.score_chunk;
@@ -453,20 +473,18 @@ static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, con
 }
 
 cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
-                             float *d_stats_part, float *d_stats, float *d_raw, float *d_gram_part, int phases,
-                             uint32_t *d_status, Profiler *prof, cudaStream_t st) {
+                             const float *d_lse, float *d_stats_part, float *d_stats, float *d_raw, float *d_gram_part,
+                             int phases, uint32_t *d_status, TmapCache *cache, Profiler *prof, cudaStream_t st) {
     CUtensorMap tq, tk;
-    cudaError_t e = make_query_tensor_map(&tq, dQw, p.units, p.rows);
-    if (e != cudaSuccess) return e;
-    e = make_key_tensor_map(&tk, p.shape, addr, dK, kTile);
+    cudaError_t e = cached_scorer_maps(cache, p, addr, dQw, dK, kTile, &tq, &tk);
     if (e != cudaSuccess) return e;
     const float c_log2 = scale * 1.4426950408889634f;
     const int MB = (p.rows + 127) / 128;
     switch (MB) {
-        case 1: return launch_scores_tc_mb<1>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
-        case 2: return launch_scores_tc_mb<2>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
-        case 3: return launch_scores_tc_mb<3>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
-        default: return launch_scores_tc_mb<4>(p, tq, tk, c_log2, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        case 1: return launch_scores_tc_mb<1>(p, tq, tk, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        case 2: return launch_scores_tc_mb<2>(p, tq, tk, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        case 3: return launch_scores_tc_mb<3>(p, tq, tk, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        default: return launch_scores_tc_mb<4>(p, tq, tk, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
     }
 }
 

@@ -33,6 +33,34 @@ struct SelSmem {
     int bin, above;
 };
 
+// What a unit may write: its slab of d_indices is offsets[u] .. offsets[u+1].  The budget should equal the slab
+// length and lie in [w, P + w]; whatever disagrees raises UNCOMP_STATUS_BOUNDS and the unit is cut to what the
+// slab and the budget both allow, so that every slot of the slab holds a valid position and nothing outside it
+// is touched: k top positions, then wn window positions, then `fill` copies of the last position.
+struct Slab {
+    int64_t begin;
+    int k, wn;
+    int64_t fill;
+};
+
+__device__ __forceinline__ Slab slab_of(const int32_t *__restrict__ budgets, const int64_t *__restrict__ offsets,
+                                        int units, int u, int P, int w, bool reporter, uint32_t *status) {
+    const int64_t o0 = offsets[u], o1 = offsets[u + 1], oend = offsets[units];
+    const int budget = budgets[u];
+    const bool off_ok = o0 >= 0 && o1 >= o0 && o1 <= oend;
+    const int64_t seg = off_ok ? o1 - o0 : 0;
+    if (!(off_ok && (int64_t)budget == seg && budget >= w && budget <= P + w) && reporter)
+        atomicOr(status, (uint32_t)UNCOMP_STATUS_BOUNDS);
+    int64_t b = min(max(budget, 0), P + w);
+    b = min(b, seg);
+    Slab s;
+    s.begin = off_ok ? o0 : 0;
+    s.k = (int)max((int64_t)0, min(b - w, (int64_t)P));
+    s.wn = (int)min((int64_t)w, b - s.k);
+    s.fill = seg - s.k - s.wn;
+    return s;
+}
+
 // Finds the bin (counting down from the top) that holds the kr-th largest element.  All threads call it.
 __device__ void find_bin(SelSmem &S, int nbins, int kr, int tid) {
     // thread t covers bins nbins-1-2t and nbins-2-2t
@@ -58,7 +86,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float *_
                                                                  int pool_kernel, int pool_mode,
                                                                  const int32_t *__restrict__ budgets,
                                                                  const int64_t *__restrict__ offsets,
-                                                                 int32_t *__restrict__ indices,
+                                                                 int units, int32_t *__restrict__ indices,
                                                                  uint32_t *__restrict__ status) {
     __shared__ SelSmem S;
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -73,14 +101,11 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float *_
         for (int t = lo; t <= hi; ++t) acc = pool_mode ? acc + r[t] : fmaxf(acc, r[t]);
         s[j] = pool_mode ? acc / (float)(hi - lo + 1) : acc;
     }
-    int budget = budgets[u];
-    if (budget < w || budget > P + w) {
-        if (tid == 0) atomicOr(status, UNCOMP_STATUS_BOUNDS);
-        budget = min(max(budget, w), P + w);
-    }
-    const int k = budget - w;
-    int32_t *out = indices + offsets[u];
-    for (int i = tid; i < w; i += kSelThreads) out[k + i] = P + i;
+    const Slab slab = slab_of(budgets, offsets, units, u, P, w, tid == 0, status);
+    const int k = slab.k;
+    int32_t *out = indices + slab.begin;
+    for (int i = tid; i < slab.wn; i += kSelThreads) out[k + i] = P + i;
+    for (int64_t i = tid; i < slab.fill; i += kSelThreads) out[k + slab.wn + i] = P + w - 1;
     if (k == 0) return;   // uniform over the CTA
     __syncthreads();      // pooled scores of this unit are visible to the whole CTA
 
@@ -153,7 +178,7 @@ constexpr int kSelCluster = 8;
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 pool_select_cluster_kernel(const float *__restrict__ raw, float *__restrict__ pooled, int P, int w, int pool_kernel,
                            int pool_mode, const int32_t *__restrict__ budgets, const int64_t *__restrict__ offsets,
-                           int32_t *__restrict__ indices, uint32_t *__restrict__ status) {
+                           int units, int32_t *__restrict__ indices, uint32_t *__restrict__ status) {
     namespace cg = cooperative_groups;
     __shared__ SelSmem S;
     __shared__ int slice_gt, slice_eq;
@@ -173,15 +198,13 @@ pool_select_cluster_kernel(const float *__restrict__ raw, float *__restrict__ po
         for (int t = lo; t <= hi; ++t) acc = pool_mode ? acc + r[t] : fmaxf(acc, r[t]);
         s[j] = pool_mode ? acc / (float)(hi - lo + 1) : acc;
     }
-    int budget = budgets[u];
-    if (budget < w || budget > P + w) {
-        if (tid == 0 && rank == 0) atomicOr(status, UNCOMP_STATUS_BOUNDS);
-        budget = min(max(budget, w), P + w);
+    const Slab slab = slab_of(budgets, offsets, units, u, P, w, tid == 0 && rank == 0, status);
+    const int k = slab.k;
+    int32_t *out = indices + slab.begin;
+    if (rank == 0) {
+        for (int i = tid; i < slab.wn; i += kSelThreads) out[k + i] = P + i;
+        for (int64_t i = tid; i < slab.fill; i += kSelThreads) out[k + slab.wn + i] = P + w - 1;
     }
-    const int k = budget - w;
-    int32_t *out = indices + offsets[u];
-    if (rank == 0)
-        for (int i = tid; i < w; i += kSelThreads) out[k + i] = P + i;
     if (k == 0) return;   // uniform over the cluster
     __syncthreads();      // this CTA reads only the pooled scores it wrote itself
 
@@ -273,10 +296,11 @@ cudaError_t launch_pool_select(const Plan &p, const float *d_raw, float *d_poole
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (p.units * kSelCluster <= 2 * sms && p.prefix >= 4096)      // few units: a cluster of CTAs per unit
         pool_select_cluster_kernel<<<p.units * kSelCluster, kSelThreads, 0, st>>>(
-            d_raw, d_pooled, p.prefix, p.shape.w, pool_kernel, pool_mode, d_budgets, d_offsets, d_indices, d_status);
+            d_raw, d_pooled, p.prefix, p.shape.w, pool_kernel, pool_mode, d_budgets, d_offsets, p.units, d_indices,
+            d_status);
     else
         pool_select_kernel<<<p.units, kSelThreads, 0, st>>>(d_raw, d_pooled, p.prefix, p.shape.w, pool_kernel, pool_mode,
-                                                            d_budgets, d_offsets, d_indices, d_status);
+                                                            d_budgets, d_offsets, p.units, d_indices, d_status);
     return cudaGetLastError();
 }
 

@@ -172,4 +172,16 @@ cudaError_t make_key_tensor_map(CUtensorMap *map, const uncomp_shape &s, const U
                                 int tile_tokens);
 cudaError_t make_query_tensor_map(CUtensorMap *map, const void *dQw, int units, int rows);
 
+// The scorer's two tensor maps as last encoded for a context.  A map depends only on the base pointer, the shape
+// and the strides, so a caller that passes the same tensors again (the two scorer calls of one pass, every pass of
+// a serving loop that reuses its buffers) pays for the encoding once.
+struct TmapCache {
+    bool k_valid, q_valid;
+    const void *k_base, *q_base;
+    UnitAddr k_addr;
+    CUtensorMap k_map, q_map;
+};
+cudaError_t cached_scorer_maps(TmapCache *cache, const Plan &p, const UnitAddr &addr, const void *dQw, const void *dK,
+                               int tile_tokens, CUtensorMap *tq, CUtensorMap *tk);
+
 }  // namespace uncomp

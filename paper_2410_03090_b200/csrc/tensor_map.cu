@@ -53,4 +53,30 @@ cudaError_t make_query_tensor_map(CUtensorMap *map, const void *dQw, int units, 
     return encode_tensor_map(map, dQw, 3, dims, str, box, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+cudaError_t cached_scorer_maps(TmapCache *cache, const Plan &p, const UnitAddr &addr, const void *dQw, const void *dK,
+                               int tile_tokens, CUtensorMap *tq, CUtensorMap *tk) {
+    TmapCache local;
+    if (!cache) { cache = &local; cache->k_valid = cache->q_valid = false; }
+    const bool same_k = cache->k_valid && cache->k_base == dK && cache->k_addr.sB == addr.sB &&
+                        cache->k_addr.sL == addr.sL && cache->k_addr.sH == addr.sH && cache->k_addr.sN == addr.sN;
+    if (!same_k) {
+        cache->k_valid = false;
+        cudaError_t e = make_key_tensor_map(&cache->k_map, p.shape, addr, dK, tile_tokens);
+        if (e != cudaSuccess) return e;
+        cache->k_base = dK;
+        cache->k_addr = addr;
+        cache->k_valid = true;
+    }
+    if (!(cache->q_valid && cache->q_base == dQw)) {
+        cache->q_valid = false;
+        cudaError_t e = make_query_tensor_map(&cache->q_map, dQw, p.units, p.rows);
+        if (e != cudaSuccess) return e;
+        cache->q_base = dQw;
+        cache->q_valid = true;
+    }
+    *tq = cache->q_map;
+    *tk = cache->k_map;
+    return cudaSuccess;
+}
+
 }  // namespace uncomp

@@ -3,6 +3,9 @@ compare with what the CUDA library produced.  The oracle never sees anything the
 except where the stage protocol says so (budgets from the GPU's erank, selection from the GPU's scores)."""
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import torch
 
@@ -11,6 +14,18 @@ from paper_2410_03090_b200 import synth
 
 ENTROPY_RTOL = 1e-4     # |dH| <= 1e-4 * max(|H_ref|, 1)
 SCORE_RTOL = 2e-3       # |d| <= 2e-3 * |ref| + 1e-12 * max_j ref
+
+
+def _map(fn, items, threads):
+    """The oracle's C functions release the interpreter lock, so units can run side by side.  Inputs are fetched
+    from the device on the calling thread."""
+    items = list(items)
+    if threads is None:
+        threads = min(len(items), os.cpu_count() or 1, 16)
+    if threads <= 1 or len(items) <= 1:
+        return [fn(*it) for it in items]
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        return list(ex.map(lambda it: fn(*it), items))
 
 
 def unit_np(t: torch.Tensor, wl: synth.Workload, u: int) -> np.ndarray:
@@ -23,13 +38,15 @@ def unit_q_np(Qw: torch.Tensor, wl: synth.Workload, u: int) -> np.ndarray:
     return Qw[b, l, h * wl.G:(h + 1) * wl.G].double().cpu().numpy()
 
 
-def check_entropy(wl, K, entropy, erank, units, k_trunc=None, center=1, norm=0):
+def check_entropy(wl, K, entropy, erank, units, k_trunc=None, center=1, norm=0, threads=None):
     k = wl.k_trunc if k_trunc is None else k_trunc
     ent = entropy.reshape(-1).double().cpu().numpy()
     er = erank.reshape(-1).double().cpu().numpy()
     worst = 0.0
-    for u in units:
-        H, E = oracle.entropy(unit_np(K, wl, u), k_trunc=k, center=bool(center), norm=norm)
+    units = list(units)
+    refs = _map(lambda X: oracle.entropy(X, k_trunc=k, center=bool(center), norm=norm),
+                [(unit_np(K, wl, u),) for u in units], threads)
+    for u, (H, E) in zip(units, refs):
         tol = ENTROPY_RTOL * max(abs(H), 1.0)
         worst = max(worst, abs(ent[u] - H) / tol)
         assert abs(ent[u] - H) <= tol, f"unit {u}: entropy {ent[u]} vs oracle {H}"
@@ -37,15 +54,24 @@ def check_entropy(wl, K, entropy, erank, units, k_trunc=None, center=1, norm=0):
     return worst
 
 
-def check_scores(wl, K, Qw, scores, units, pool_kernel=None, pool_mode=None, scale=None):
+def oracle_lse(wl, K, Qw, units, scale=None, threads=None) -> dict:
+    """{unit: [G, w] fp64 log-sum-exp of its window rows} from the oracle."""
+    units = list(units)
+    refs = _map(lambda Q, X: oracle.window_lse(Q, X, scale), [(unit_q_np(Qw, wl, u), unit_np(K, wl, u)) for u in units],
+                threads)
+    return dict(zip(units, refs))
+
+
+def check_scores(wl, K, Qw, scores, units, pool_kernel=None, pool_mode=None, scale=None, threads=None):
     pk = wl.pool_kernel if pool_kernel is None else pool_kernel
     pm = wl.pool_mode if pool_mode is None else pool_mode
     P = wl.N - wl.w
     sc = scores.reshape(-1, P)
     worst = 0.0
-    for u in units:
-        raw = oracle.window_scores(unit_q_np(Qw, wl, u), unit_np(K, wl, u), scale)
-        ref = oracle.pool(raw, pk, pm)
+    units = list(units)
+    refs = _map(lambda Q, X: oracle.pool(oracle.window_scores(Q, X, scale), pk, pm),
+                [(unit_q_np(Qw, wl, u), unit_np(K, wl, u)) for u in units], threads)
+    for u, ref in zip(units, refs):
         got = sc[u].double().cpu().numpy()
         tol = SCORE_RTOL * np.abs(ref) + 1e-12 * ref.max()
         err = np.abs(got - ref) / tol

@@ -240,13 +240,85 @@ def test_host_side_rejections_and_status_word():
     # device-side conditions arrive through the status word and leave the context usable
     ub.uncomp_entropy(ctx, K, max_iters=1)
     assert ub.uncomp_status(ctx) & ub.UNCOMP_STATUS_NOT_CONVERGED
-    bad = b.clone()
-    bad[0, 0, 0] = wl.N + 5
-    ub.uncomp_score_select(ctx, Qw, K, bad, o, wl.units * 100)
-    assert ub.uncomp_status(ctx) & ub.UNCOMP_STATUS_BOUNDS
     ent, _ = ub.uncomp_entropy(ctx, K)
     assert ub.uncomp_status(ctx) == 0
     parity.check_entropy(wl, K, ent, _, [0, 5])
+
+
+@pytest.mark.parametrize("unit,value", [(3, "N+5"), (7, "N+5"), (7, "w-3"), (4, "0"), (2, "50"), (0, "-9")])
+def test_bad_budget_stays_inside_its_slab(unit, value):
+    # A budget that disagrees with its slab (too large, below the window, negative, or just different) is reported
+    # and cut to the slab; the last unit is the one that would run off the end of d_indices.  The index buffer has
+    # a guard region behind it that no case may touch, and it is sized so that even a unit writing N entries from
+    # its offset would stay inside the allocation.
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=512, L=1)
+    K, V, Qw = synth.generate(wl, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    er = torch.ones(wl.B, wl.L, wl.H, device="cuda")
+    b, o, _, _ = ub.uncomp_assign_budgets(ctx, er, 100, 1, 100)
+    total = wl.units * 100
+    buf = torch.full((total + 2 * wl.N,), -7, dtype=torch.int32, device="cuda")
+    scores = torch.empty(wl.B, wl.L, wl.H, wl.N - wl.w, device="cuda")
+    bad = b.clone()
+    bad.view(-1)[unit] = {"N+5": wl.N + 5, "w-3": wl.w - 3, "0": 0, "50": 50, "-9": -9}[value]
+    ub.uncomp_score_select(ctx, Qw, K, bad, o, total, scores=scores, indices=buf[:total])
+    assert ub.uncomp_status(ctx) == ub.UNCOMP_STATUS_BOUNDS
+    assert bool((buf[total:] == -7).all())
+    idx = buf[:total]
+    parity.check_select(wl, scores, b, o, idx, [u for u in range(wl.units) if u != unit])
+    slab = idx[unit * 100:(unit + 1) * 100].cpu().numpy()
+    assert slab.min() >= 0 and slab.max() <= wl.N - 1          # every slot holds a valid position
+    want = min(max(int(bad.view(-1)[unit]), 0), 100)
+    if want >= wl.w:                                           # as much of the selection as budget and slab allow
+        import oracle
+        ref = oracle.select(scores.view(wl.units, -1)[unit].double().cpu().numpy(), wl.w, want)
+        np.testing.assert_array_equal(slab[:want], ref)
+    assert (slab[want:] == wl.N - 1).all()
+    # the compaction of such a slab reads valid rows only
+    Kc, Vc = ub.uncomp_compact(ctx, K, V, idx, o, total)
+    assert ub.uncomp_status(ctx) == 0
+    parity.check_compact(wl, K, V, idx, o, Kc, Vc, [unit])
+
+
+def test_bad_offsets_write_nothing_outside_and_bad_indices_are_clamped():
+    ub = _ub()
+    wl = synth.scaled(synth.WORKLOADS["c2"], N=512, L=1)
+    K, V, Qw = synth.generate(wl, "cuda")
+    ctx = ub.Context(ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype))
+    er = torch.ones(wl.B, wl.L, wl.H, device="cuda")
+    b, o, _, _ = ub.uncomp_assign_budgets(ctx, er, 100, 1, 100)
+    total = wl.units * 100
+    scores = torch.empty(wl.B, wl.L, wl.H, wl.N - wl.w, device="cuda")
+    for case in ("shifted", "negative", "beyond_end"):
+        o2 = o.clone()
+        if case == "shifted":
+            o2[5] = 450                  # unit 4 gets 50 slots for a budget of 100, unit 5 gets 150
+        elif case == "negative":
+            o2[0] = -300
+        else:
+            o2[7] = total + 40           # unit 6 would end, and unit 7 start, beyond offsets[units]
+        buf = torch.full((total + 2 * wl.N,), -7, dtype=torch.int32, device="cuda")
+        ub.uncomp_score_select(ctx, Qw, K, b, o2, total, scores=scores, indices=buf[:total])
+        assert ub.uncomp_status(ctx) == ub.UNCOMP_STATUS_BOUNDS, case
+        assert bool((buf[total:] == -7).all()), case
+        touched = {"shifted": (4, 5), "negative": (0,), "beyond_end": (6, 7)}[case]
+        parity.check_select(wl, scores, b, o, buf[:total], [u for u in range(wl.units) if u not in touched])
+        written = buf[:total][buf[:total] != -7]
+        assert int(written.min()) >= 0 and int(written.max()) <= wl.N - 1, case
+    # compaction: an index outside [0, N) is replaced by the nearest valid row and reported
+    idx = ub.uncomp_score_select(ctx, Qw, K, b, o, total, scores=scores)
+    assert ub.uncomp_status(ctx) == 0
+    Kc0, Vc0 = ub.uncomp_compact(ctx, K, V, idx, o, total)
+    hurt = idx.clone()
+    hurt[250], hurt[251] = -1, wl.N                      # rows 50 and 51 of unit 2
+    Kc, Vc = ub.uncomp_compact(ctx, K, V, hurt, o, total)
+    assert ub.uncomp_status(ctx) == ub.UNCOMP_STATUS_BOUNDS
+    keep = torch.ones(total, dtype=torch.bool, device="cuda")
+    keep[250:252] = False
+    assert torch.equal(Kc[keep], Kc0[keep]) and torch.equal(Vc[keep], Vc0[keep])
+    assert torch.equal(Kc[250], K[0, 0, 2, 0]) and torch.equal(Kc[251], K[0, 0, 2, wl.N - 1])
+    assert torch.equal(Vc[250], V[0, 0, 2, 0]) and torch.equal(Vc[251], V[0, 0, 2, wl.N - 1])
 
 
 def _gram_oracle(K_unit_np):

@@ -18,7 +18,7 @@ from paper_2410_03090_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def _compare(ub, wl):
+def _compare(ub, wl, tol=2e-6):
     K, _, _ = synth.generate(wl, "cuda")
     shape = ub.make_shape(wl.B, wl.L, wl.H, wl.Hq, wl.N, wl.d, wl.w, wl.dtype)
     ctx = ub.Context(shape)
@@ -28,9 +28,11 @@ def _compare(ub, wl):
     torch.cuda.synchronize()
     assert ub.uncomp_status(ctx) == 0
     scale = ref[:, :128 * 128].abs().amax(dim=1, keepdim=True)
-    # same kernels, same summation order: the tolerance of the Gram tests (2e-6 of the largest entry)
-    assert float(((out - ref).abs() / scale).max()) <= 2e-6
+    # same kernels and, for these shapes, the same token chunks as uncomp_gram: the tolerance of the Gram tests
+    # (2e-6 of the largest entry); a caller with longer chunks passes its own
+    assert float(((out - ref).abs() / scale).max()) <= tol
     assert torch.isfinite(out).all()
+    return out
 
 
 def test_gram_static_matches_workspace_entry_point_twice_in_a_row():
@@ -41,6 +43,38 @@ def test_gram_static_matches_workspace_entry_point_twice_in_a_row():
     _compare(ub, small)
     fp32 = synth.WORKLOADS["c1"]                                      # fp32 keys take the fp64 partials
     _compare(ub, fp32)
+
+
+def test_gram_static_is_exact_on_integer_keys_against_the_oracle():
+    # integer-valued keys: every product and partial sum is exact, so the result must equal the oracle's X^T X and
+    # column sums bit for bit whatever the chunking; the second shape needs the longer chunks (8 units x 17 chunks
+    # of 1024 tokens would not fit the array)
+    import oracle
+    from paper_2410_03090_b200 import binding as ub
+    for units, N in ((3, 1000), (8, 17000)):
+        g = torch.Generator(device="cuda").manual_seed(N)
+        K = torch.randint(-3, 4, (1, 1, units, N, 128), generator=g, device="cuda").to(torch.bfloat16)
+        K[0, 0, units - 1, N - 1, :] = 5.0
+        shape = ub.make_shape(1, 1, units, units, N, 128, 8, "bf16")
+        out = torch.full((units, 128 * 128 + 128), float("nan"), dtype=torch.float64, device="cuda")
+        ub.uncomp_gram_static(shape, K, out)
+        torch.cuda.synchronize()
+        for u in (0, units - 1):
+            X = K[0, 0, u].double().cpu().numpy()
+            got = out[u].cpu().numpy()
+            np.testing.assert_array_equal(got[:128 * 128].reshape(128, 128), oracle.covariance(X, center=False))
+            np.testing.assert_array_equal(got[128 * 128:], X.sum(axis=0))
+
+
+def test_gram_static_at_its_documented_maximum():
+    # one layer of the 32K-token workload: 8 heads x 32768 tokens, 64 partials of 4096 tokens each
+    from paper_2410_03090_b200 import binding as ub
+    # (uncomp_gram takes 1024: fp32 accumulation on the tensor cores over four times as many tokens per partial
+    # rounds more, measured 1e-5 of the largest entry)
+    wl = synth.scaled(synth.WORKLOADS["c3"], L=1)
+    _compare(ub, wl, tol=4e-5)
+    wl64 = synth.scaled(synth.WORKLOADS["c2"], N=512, L=8)            # 64 units, one partial each
+    _compare(ub, wl64)
 
 
 def test_gram_static_refuses_shapes_beyond_its_array():
