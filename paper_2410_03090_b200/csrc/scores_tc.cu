@@ -11,15 +11,16 @@
 // K tiles (128 tokens x 128 features, two 128B-swizzled boxes of 64 features) stream through a TMA ring;
 // the unit's window queries stay in shared memory for the whole CTA.  Both operands are K-major.
 //
-// CTA = 576 threads on one SM: warps 0-15 softmax in two groups of eight that take alternate token tiles
-// (so the four warps of an SM sub-partition are in different phases: while one group waits for its
-// accumulator, the other keeps the exponential unit busy); inside a group warp % 4 selects the TMEM lane
-// quarter and bit 2 of the warp index the 64-column half of an accumulator.  Warp 16 is the TMA producer,
-// warp 17 allocates TMEM and issues the MMAs.  Each group owns two of the four 128-column accumulators.
+// CTA on one SM: warps 0-15 softmax in two groups of eight that take alternate token tiles (so the four
+// warps of an SM sub-partition are in different phases: while one group waits for its accumulator, the
+// other keeps the exponential unit busy); inside a group warp % 4 selects the TMEM lane quarter and bit 2
+// of the warp index the 64-column half of an accumulator.  Warp 16 is the TMA producer, warp 17 allocates
+// TMEM and issues the MMAs.  The 128-column accumulators form one ring that both groups draw from in item
+// order (item = one 128-row block of one tile): four buffers in modes 0 and 1, three in mode 2.
 // Mode 2 of the kernel is pass A with the Gram stage folded in: the K tile that is in shared memory for
-// Qw K^T is also the MN-major operand of G += K_tile^T K_tile (and of the narrow all-ones MMA for the column
-// sums), so the entropy stage costs no second sweep over K.  The tensor pipe has the room (pass A is bound
-// by the exponential unit); TMEM then holds one accumulator per softmax group plus the Gram block.
+// Qw K^T is also the MN-major operand of G += K_tile^T K_tile, so the entropy stage costs no second sweep
+// over K.  The Gram block takes the last 128 TMEM columns; the column sums s = K^T 1 are added up by two
+// extra warps (18, 19) with plain global loads of the same tokens (L2 hits), in a fixed order.
 // Every wait is bounded; a timeout raises UNCOMP_STATUS_TIMEOUT and the CTA drains and exits.
 #include "tc_common.cuh"
 
@@ -31,17 +32,18 @@ constexpr int kHalfBytes = 128 * 128;            // 64 features x 128 rows/token
 constexpr int kBlockBytes = 2 * kHalfBytes;      // one K tile or one block of 128 query rows
 constexpr int kNB = 4;                           // accumulator buffers (x 128 TMEM columns = all 512)
 constexpr int kSoftThreads = 512;
-constexpr int kScoreThreads = kSoftThreads + 64;
+constexpr int kScoreThreads = kSoftThreads + 64;  // modes 0 and 1
+constexpr int kGramThreads = kScoreThreads + 64;  // mode 2: two more warps for the column sums
 constexpr int kMaxStages = 4;
 
 struct ScoreTail {
-    uint64_t full[kMaxStages], empty[kMaxStages], qfull, tfull[kNB], tempty[kNB], gfull;
+    uint64_t full[kMaxStages], empty[kMaxStages], qfull, tfull[2 * kNB], tempty[kNB], gfull;
     uint32_t tmem_base;
 };
 
 __host__ __device__ constexpr int score_stages(int MB) { return MB <= 2 ? 4 : (MB == 3 ? 3 : 2); }
 __host__ __device__ constexpr int score_smem(int MB) {
-    return 1024 + MB * kBlockBytes + score_stages(MB) * kBlockBytes + MB * 128 * 4 + 2 * 4 * 128 * 4 + 2048 +
+    return 1024 + MB * kBlockBytes + score_stages(MB) * kBlockBytes + MB * 128 * 4 + 2 * 4 * 128 * 4 +
            (int)sizeof(ScoreTail);
 }
 
@@ -52,6 +54,22 @@ __device__ __forceinline__ float ex2(float x) {
 }
 __device__ __forceinline__ void all_soft_barrier() { asm volatile("bar.sync 3, 512;" ::: "memory"); }
 __device__ __forceinline__ void group_barrier(int g) { asm volatile("bar.sync %0, 256;" ::"r"(1 + g) : "memory"); }
+__device__ __forceinline__ void sum_warps_barrier() { asm volatile("bar.sync 4, 64;" ::: "memory"); }
+__device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+__device__ __forceinline__ void add_bf16x8(float (&acc)[8], const uint4 &x) {
+    acc[0] += bf16_lo(x.x); acc[1] += bf16_hi(x.x);
+    acc[2] += bf16_lo(x.y); acc[3] += bf16_hi(x.y);
+    acc[4] += bf16_lo(x.z); acc[5] += bf16_hi(x.z);
+    acc[6] += bf16_lo(x.w); acc[7] += bf16_hi(x.w);
+}
+// 16-byte read-only global load that does not allocate in L1
+__device__ __forceinline__ uint4 ld_stream16(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -105,14 +123,19 @@ __device__ __forceinline__ float colsum_partial(const uint32_t (&v)[64], float c
 }  // namespace
 
 template <int MB, int MODE>   // MODE 0: pass A, 1: pass B, 2: pass A fused with the Gram stage
-__global__ void __launch_bounds__(kScoreThreads, 1)
+__global__ void __launch_bounds__(kGramThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant__ CUtensorMap tmapK, int L, int H,
                 int N, int w, int rows, int chunk, int splits, float c_log2, float *__restrict__ stats_part,
                 const float *__restrict__ mprime, float *__restrict__ raw, float *__restrict__ gram_part,
-                uint32_t *__restrict__ status) {
+                const void *__restrict__ Kraw, const UnitAddr kaddr, uint32_t *__restrict__ status) {
     constexpr bool PASS_B = MODE == 1, GRAM = MODE == 2;
-    constexpr int NA = GRAM ? 1 : 2;                 // accumulators per softmax group
-    constexpr uint32_t kGramCol = 256, kSumCol = 384;  // TMEM columns of the Gram block and the column sums
+    constexpr int NB = GRAM ? 3 : kNB;               // accumulator ring: item n lives in buffer n % NB
+    // "Item n is ready" is signalled on barrier n % (2 NB): a softmax group that waits for the first item of its
+    // next tile may get there before the other group's item n - NB has completed, and with one barrier per buffer
+    // the parity of that unfinished phase could not be told from the one waited for.  The user of this barrier
+    // before item n is item n - 2 NB, which lies in a tile this group has already consumed (2 NB > MB).
+    constexpr int NF = 2 * NB;
+    constexpr uint32_t kGramCol = 384;               // TMEM columns of the Gram block (mode 2)
     constexpr int S = score_stages(MB);
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = tc::smem_u32(smem_raw);
@@ -122,8 +145,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
     const uint32_t k_addr = q_addr + MB * kBlockBytes;
     float *mp = reinterpret_cast<float *>(smem + (MB + S) * kBlockBytes);      // [MB * 128]
     float *colsum = mp + MB * 128;                                             // [2][4][128]
-    unsigned char *ones = reinterpret_cast<unsigned char *>(colsum + 2 * 4 * 128);   // 2 KB, mode 2 only
-    ScoreTail &T = *reinterpret_cast<ScoreTail *>(ones + 2048);
+    ScoreTail &T = *reinterpret_cast<ScoreTail *>(colsum + 2 * 4 * 128);
 
     const int c = blockIdx.x, u = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -141,15 +163,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
         }
         tc::mbar_init(tc::smem_u32(&T.qfull), 1);
         tc::mbar_init(tc::smem_u32(&T.gfull), 1);
-        for (int i = 0; i < kNB; ++i) {
-            tc::mbar_init(tc::smem_u32(&T.tfull[i]), 1);
-            tc::mbar_init(tc::smem_u32(&T.tempty[i]), kSoftThreads / 64);   // the 8 warps of one group
-        }
+        for (int i = 0; i < 2 * kNB; ++i) tc::mbar_init(tc::smem_u32(&T.tfull[i]), 1);
+        for (int i = 0; i < kNB; ++i) tc::mbar_init(tc::smem_u32(&T.tempty[i]), kSoftThreads / 64);   // the 8 warps of one group
         tc::fence_mbar_init();
-    }
-    if (GRAM) {   // all-ones bf16 operand of the column-sum MMA
-        for (int i = threadIdx.x; i < 2048 / 4; i += kScoreThreads) reinterpret_cast<uint32_t *>(ones)[i] = 0x3f803f80u;
-        tc::fence_proxy_async();
     }
     if (warp == 17) {
         tc::tmem_alloc(tc::smem_u32(&T.tmem_base), 512);
@@ -205,15 +221,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
             for (int mb = 0; mb < MB; ++mb) q_lo[mb] = tc::desc_lo(d0) + (uint32_t)(mb * kBlockBytes >> 4);
             const uint32_t k_lo0 = tc::desc_lo(tc::smem_desc_sw128(k_addr, 16, 1024));
             const uint64_t gd = tc::smem_desc_sw128(k_addr, kHalfBytes, 1024);
-            const uint64_t od = tc::smem_desc_sw128(tc::smem_u32(ones), 1024, 1024);
-            const uint32_t g_lo0 = tc::desc_lo(gd), g_hi = tc::desc_hi(gd), ones_lo = tc::desc_lo(od), ones_hi = tc::desc_hi(od);
+            const uint32_t g_lo0 = tc::desc_lo(gd), g_hi = tc::desc_hi(gd);
             // Mode 2: the Gram MMAs of a tile only have to be issued before its stage is handed back, so they
             // are deferred by up to one tile and issued while this thread would otherwise wait for an
             // accumulator: the latency-critical QK^T MMAs never queue behind them.
             int g_done = 0;                    // tiles whose Gram MMAs are issued (and whose stage is released)
             auto issue_gram = [&](int t) {
                 constexpr uint32_t idesc_g = tc::idesc_bf16_f32(128, 128, 1, 1);
-                constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, 16, 1, 1);
                 const int sg = t % S;
                 const uint32_t g_lo = g_lo0 + (uint32_t)(sg * (kBlockBytes >> 4));
 #pragma unroll
@@ -222,7 +236,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                     // apart); 16 tokens further = +128 address units
                     const uint32_t acc = (t > 0 || k > 0) ? 1u : 0u;
                     tc::mma_f16_ss_lohi(tmem + kGramCol, g_lo + k * 128, g_lo + k * 128, g_hi, idesc_g, acc);
-                    tc::mma_f16_ss2(tmem + kSumCol, g_lo + k * 128, g_hi, ones_lo, ones_hi, idesc_s, acc);
                 }
                 tc::mma_commit(tc::smem_u32(&T.empty[sg]));
             };
@@ -234,11 +247,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                 const uint32_t k_lo = k_lo0 + (uint32_t)(s * (kBlockBytes >> 4));
 #pragma unroll
                 for (int mb = 0; mb < MB; ++mb) {
-                    // tile i belongs to softmax group i & 1, which owns NA accumulators of 128 columns
-                    const int lq = (i >> 1) * MB + mb, buf = NA * (i & 1) + (lq % NA);
-                    if (ok && lq >= NA) {
+                    // item n (tile i, row block mb) goes to ring buffer n % NB, once item n - NB has been drained
+                    const int n = i * MB + mb, buf = n % NB;
+                    if (ok && n >= NB) {
                         const uint32_t bar = tc::smem_u32(&T.tempty[buf]);
-                        const uint32_t parity = ((lq / NA) - 1) & 1;
+                        const uint32_t parity = ((n / NB) - 1) & 1;
                         if (GRAM) {
                             uint32_t spins = 0;
                             while (!tc::mbar_try_wait(bar, parity)) {
@@ -262,7 +275,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                         if (PASS_B) tc::mma_f16_ss_lohi(d_tmem, k_lo + off, q_lo[mb] + off, dhi, idesc, k > 0);
                         else tc::mma_f16_ss_lohi(d_tmem, q_lo[mb] + off, k_lo + off, dhi, idesc, k > 0);
                     }
-                    tc::mma_commit(tc::smem_u32(&T.tfull[buf]));
+                    tc::mma_commit(tc::smem_u32(&T.tfull[n % NF]));
                 }
                 if (!ok) break;
                 if (GRAM) {
@@ -274,6 +287,42 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
             if (GRAM) {
                 if (ok) while (g_done < ntiles) issue_gram(g_done++);
                 tc::mma_commit(tc::smem_u32(&T.gfull));
+            }
+        }
+    } else if (warp >= 18) {
+        // ---------------- column sums s = K^T 1 (mode 2 only) ----------------
+        // Two warps add up the CTA's token chunk with plain 16-byte global loads (the lines are in L2: the TMA
+        // stream fetches the same tokens), so the shared-memory banks stay with the MMA operands and the sums
+        // need no place in the tile pipeline.  A lane owns one 16-byte chunk (8 features) of the 256-byte row and
+        // one of four row phases; its rows are added in increasing order, the phases in a fixed order below.
+        if (GRAM) {
+            const int sw = warp - 18, ch = lane & 15, phase = 2 * sw + (lane >> 4);
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            const unsigned char *rowp = reinterpret_cast<const unsigned char *>(Kraw) +
+                                        2 * (kaddr.base(u) + (int64_t)(t0 + phase) * kaddr.sN) + 16 * ch;
+            const int64_t step = 2 * 4 * kaddr.sN;                 // four rows further, in bytes
+            const int nrows = t1 > t0 + phase ? (t1 - t0 - phase + 3) / 4 : 0;
+            int r = 0;
+            for (; r + 16 <= nrows; r += 16) {          // 16 loads in flight per lane cover the L2 latency
+                uint4 x[16];
+#pragma unroll
+                for (int q = 0; q < 16; ++q) x[q] = ld_stream16(rowp + (int64_t)(r + q) * step);
+#pragma unroll
+                for (int q = 0; q < 16; ++q) add_bf16x8(acc, x[q]);
+            }
+            for (; r < nrows; ++r) add_bf16x8(acc, ld_stream16(rowp + (int64_t)r * step));
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);   // phases 2 sw, 2 sw + 1
+            float *xch = colsum;                               // unused by the softmax warps in this mode
+            if (sw == 1 && lane < 16) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) xch[ch * 8 + e] = acc[e];
+            }
+            sum_warps_barrier();
+            if (sw == 0 && lane < 16 && ntiles > 0) {
+                float *out = gram_part + ((size_t)u * splits + c) * (kD * kD + kD) + kD * kD;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) out[ch * 8 + e] = acc[e] + xch[ch * 8 + e];
             }
         }
     } else {
@@ -297,10 +346,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
             float acc = 0.f;
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
-                const int lq = (i >> 1) * MB + mb, buf = NA * group + (lq % NA);
+                const int n = i * MB + mb, buf = n % NB;
                 uint32_t v[64];
                 if (!dead) {
-                    const bool ok = tc::mbar_wait(tc::smem_u32(&T.tfull[buf]), (lq / NA) & 1, status);
+                    const bool ok = tc::mbar_wait(tc::smem_u32(&T.tfull[n % NF]), (n / NF) & 1, status);
                     dead = !__all_sync(0xffffffffu, ok);
                 }
                 if (!dead) {
@@ -384,11 +433,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                 for (int q4 = 0; q4 < 8; ++q4)
                     dst[q4] = make_float4(__uint_as_float(r[4 * q4]), __uint_as_float(r[4 * q4 + 1]),
                                           __uint_as_float(r[4 * q4 + 2]), __uint_as_float(r[4 * q4 + 3]));
-                if (cb == 0) {
-                    tc::tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + kSumCol, r);   // only column 0 is used
-                    tc::tmem_ld_wait();
-                    out[kD * kD + lane_row] = __uint_as_float(r[0]);
-                }
             }
         }
     }
@@ -430,7 +474,8 @@ static cudaError_t raise_smem_limit_once() {
 }
 
 template <int MB>
-static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, const CUtensorMap &tk, float c_log2,
+static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, const CUtensorMap &tk, const void *dK,
+                                       const UnitAddr &addr, float c_log2,
                                        const float *d_lse, float *d_stats_part, float *d_mprime, float *d_raw,
                                        float *d_gram_part, int phases, uint32_t *d_status, Profiler *prof,
                                        cudaStream_t st) {
@@ -442,13 +487,13 @@ static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, con
         ProfScope ps(prof, d_gram_part ? kSlotGramStats : kSlotScoreStats, st);
         dim3 grid(p.score_splits, p.units);
         if (d_gram_part)
-            score_tc_kernel<MB, 2><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
+            score_tc_kernel<MB, 2><<<grid, kGramThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
                                                                       p.score_splits, c_log2, d_stats_part, nullptr,
-                                                                      nullptr, d_gram_part, d_status);
+                                                                      nullptr, d_gram_part, dK, addr, d_status);
         else
             score_tc_kernel<MB, 0><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
                                                                       p.score_splits, c_log2, d_stats_part, nullptr,
-                                                                      nullptr, nullptr, d_status);
+                                                                      nullptr, nullptr, nullptr, addr, d_status);
     }
     if (phases & kScorePhaseColsum) {
         {
@@ -467,7 +512,7 @@ static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, con
         dim3 grid(splitsB, p.units);
         score_tc_kernel<MB, 1><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
                                                                   splitsB, c_log2, nullptr, d_mprime, d_raw, nullptr,
-                                                                  d_status);
+                                                                  nullptr, addr, d_status);
     }
     return cudaGetLastError();
 }
@@ -481,10 +526,10 @@ cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, con
     const float c_log2 = scale * 1.4426950408889634f;
     const int MB = (p.rows + 127) / 128;
     switch (MB) {
-        case 1: return launch_scores_tc_mb<1>(p, tq, tk, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
-        case 2: return launch_scores_tc_mb<2>(p, tq, tk, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
-        case 3: return launch_scores_tc_mb<3>(p, tq, tk, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
-        default: return launch_scores_tc_mb<4>(p, tq, tk, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        case 1: return launch_scores_tc_mb<1>(p, tq, tk, dK, addr, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        case 2: return launch_scores_tc_mb<2>(p, tq, tk, dK, addr, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        case 3: return launch_scores_tc_mb<3>(p, tq, tk, dK, addr, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
+        default: return launch_scores_tc_mb<4>(p, tq, tk, dK, addr, c_log2, d_lse, d_stats_part, d_stats, d_raw, d_gram_part, phases, d_status, prof, st);
     }
 }
 
