@@ -24,14 +24,61 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes per (unit x token) of one launch, dram__bytes_read.sum + dram__bytes_write.sum from the ncu capture
-# summarised in profiles/kernels_c3_N16384_L10_ncu_full.md (80 units x 16384 tokens; traffic grows with
-# units x tokens, so a full-size launch is scaled by that product).  Set to None when a kernel changes.
-TRAFFIC_PER_UNIT_TOKEN = {"gram_score_stats": (341.02e6 + 33.73e6) / (80 * 16384),
-                          "score_colsum": (340.94e6 + 7.60e6) / (80 * 16384)}
+# Hardware counters of the two scorer kernels from one ncu capture of a smaller case of the same workload
+# (80 units x 16384 tokens): DRAM bytes per (unit x token) of one launch (dram__bytes_read.sum +
+# dram__bytes_write.sum; traffic grows with units x tokens, so a full-size launch is scaled by that product),
+# tensor-pipe and exponential-unit (XU) activity in % of peak.  They describe the kernel source whose SHA-256 is
+# recorded beside them: when the file has changed since the capture, the bench prints null instead.
+NCU_COUNTERS = {
+    "source": "paper_2410_03090_b200/csrc/scores_tc.cu",
+    "sha256": "",
+    "capture": "",
+    "kernels": {},
+}
 EXP_KERNELS = ("score_stats", "score_colsum", "gram_score_stats")
 METRIC = "compression_pass_tokens_per_s"
 UNIT = "tokens/s"
+
+
+def ncu_counters(kernel):
+    """Counters recorded for `kernel`, or None when there are none or the kernel source has changed since."""
+    import hashlib
+    ent = NCU_COUNTERS["kernels"].get(kernel)
+    if not ent or not NCU_COUNTERS["sha256"]:
+        return None
+    try:
+        with open(os.path.join(ROOT, NCU_COUNTERS["source"]), "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    return ent if digest == NCU_COUNTERS["sha256"] else None
+
+
+def tensor_peak(peaks, clocks, timed_s):
+    """Which measured bf16 peak a kernel timed inside this run is held against.  The burst figure applies to a
+    short timed region that ran at full clocks with no power cap; once the region lasts a second or more, or
+    the clock record shows sw_power_cap, the GPU is in the regime the sustained figure was taken in."""
+    capped = "sw_power_cap" in (clocks.get("reasons") or [])
+    if timed_s < 1.0 and not capped:
+        return peaks["bf16_burst"], "burst bf16"
+    return peaks["bf16_sustained"], "sustained bf16"
+
+
+def composite_bound(wl, qk_passes, hbm_gbs, tensor_tflops, sm_count, sm_mhz, ms_step):
+    """Lower bounds of one pass of the whole workload and the fraction of the largest the pass reaches:
+    t_hbm (algorithmic bytes at the copy peak), t_tensor (Gram + qk_passes window products at the bf16 peak),
+    t_exp (qk_passes x rows x tokens exponentials at 16 per clock per SM)."""
+    u, N, d, rows = wl.units, wl.N, wl.d, wl.G * wl.w
+    flops = u * (2.0 * N * d * d + qk_passes * 2.0 * rows * d * N)
+    exps = u * qk_passes * float(rows) * N
+    t_hbm = wl.algorithmic_bytes() / (hbm_gbs * 1e9) * 1e3
+    t_tensor = flops / (tensor_tflops * 1e12) * 1e3
+    t_exp = exps / (sm_count * 16.0 * sm_mhz * 1e6) * 1e3
+    t_min = max(t_hbm, t_tensor, t_exp)
+    return {"qk_passes": qk_passes, "t_hbm_ms": round(t_hbm, 4), "t_tensor_ms": round(t_tensor, 4),
+            "t_exp_ms": round(t_exp, 4), "t_min_ms": round(t_min, 4),
+            "binding": "hbm" if t_min == t_hbm else ("tensor" if t_min == t_tensor else "exp"),
+            "frac_of_t_min": round(t_min / ms_step, 4) if ms_step else None}
 
 
 def _peaks():
@@ -103,13 +150,15 @@ class ClockSampler(threading.Thread):
 
 
 # ------------------------------------------------------------------------------------- roofline per kernel
-def kernel_specs(wl, peaks, sustained: bool, D=None, n_keep=None, cache_rows=None):
+def kernel_specs(wl, peaks, sustained, D=None, n_keep=None, cache_rows=None):
     """Algorithmic work of one launch of each kernel of the pass (units of one rank).  D and n_keep (width of
     a hidden-state row, tokens kept) size the kernels of the hidden-state eviction step; without them those
     entries carry no work figure."""
     u, N, d, P = wl.units, wl.N, wl.d, wl.N - wl.w
     rows, s = wl.G * wl.w, wl.elem_bytes
-    tens = peaks["bf16_sustained"] if sustained else peaks["bf16_burst"]
+    # `sustained`: True / False pick one of the measured bf16 peaks, a number is taken as the peak itself
+    tens = float(sustained) if not isinstance(sustained, bool) else (
+        peaks["bf16_sustained"] if sustained else peaks["bf16_burst"])
     if wl.dtype == "fp32":
         tens = tens / 2.0 / 16.0   # fp32 inputs run on the CUDA cores; no tensor peak applies
     hbm = peaks["hbm_gbs"]
@@ -211,6 +260,23 @@ def run_reference(args):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def prefill_lse(wl, K, Qw):
+    """[B, L, Hq, w] float32: the natural-log sum of exponentials of every window row's scaled, causally visible
+    logits.  Stands in for what the prefill attention kernel keeps per row; an input of the timed call."""
+    import torch
+    P = wl.N - wl.w
+    out = torch.empty(wl.B, wl.L, wl.Hq, wl.w, dtype=torch.float32, device=K.device)
+    pos = torch.arange(wl.N, device=K.device)[None, :]
+    hidden = (pos > (P + torch.arange(wl.w, device=K.device))[:, None])[None]
+    for b in range(wl.B):
+        for l in range(wl.L):
+            for h in range(wl.H):
+                q = Qw[b, l, h * wl.G:(h + 1) * wl.G].float()
+                s = torch.einsum("gwd,nd->gwn", q, K[b, l, h].float()) / wl.d ** 0.5
+                out[b, l, h * wl.G:(h + 1) * wl.G] = torch.logsumexp(s.masked_fill(hidden, float("-inf")), dim=-1)
+    return out
 
 
 def _workload_name(wl):
@@ -742,8 +808,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale-N", type=int, default=0, help="profiling aid: same recipe at a shorter sequence")
     ap.add_argument("--scale-L", type=int, default=0, help="profiling aid: same recipe with fewer layers")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-lse", action="store_true", help="skip the second timed run with caller-supplied log-sum-exp")
     ap.add_argument("--path", default="kv", choices=["kv", "hidden", "decode", "prepare", "wide"],
                     help="kv: the KV-cache compression pass (the default and the headline); hidden: the "
                          "hidden-state eviction of one layer-group boundary; decode: one decode-time update of "
@@ -800,65 +867,99 @@ def main():
         if world > 1:
             dist.barrier()
 
-    for _ in range(args.warmup):
-        cp.run(K, V, Qw)
-    torch.cuda.synchronize()
-    assert cp.status() == 0
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
 
-    sampler = ClockSampler(local)
-    sampler.start()
-    ub.uncomp_profile_enable(cp.ctx, True)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    torch.cuda.synchronize()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        cp.run(K, V, Qw)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    barrier()
-    clocks = sampler.stop()
-    ms_total = ev0.elapsed_time(ev1)
-    prof = ub.uncomp_profile_read(cp.ctx)
-    ub.uncomp_profile_enable(cp.ctx, False)
-    ms_total = shard.max_over_ranks(ms_total, dev, world)
-    ms_step = ms_total / args.steps
+    def timed_passes(lse):
+        """W warm-up and K timed passes (barrier + synchronize on both sides, CUDA events on the launching stream,
+        max over ranks); returns the step time, the clock record and the per-kernel event times."""
+        for _ in range(args.warmup):
+            cp.run(K, V, Qw, lse=lse)
+        torch.cuda.synchronize()
+        assert cp.status() == 0
+        sampler = ClockSampler(local)
+        sampler.start()
+        ub.uncomp_profile_enable(cp.ctx, True)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for _ in range(args.steps):
+            cp.run(K, V, Qw, lse=lse)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+        clk = sampler.stop()
+        ms_total = ev0.elapsed_time(ev1)
+        prof_ = ub.uncomp_profile_read(cp.ctx)
+        ub.uncomp_profile_enable(cp.ctx, False)
+        return shard.max_over_ranks(ms_total, dev, world) / args.steps, clk, prof_
+
+    def kernel_records(prof_, clk, ms_step_):
+        """Per-kernel roofline entries from the events the library recorded inside the timed region."""
+        tens, tens_name = tensor_peak(peaks, clk, ms_step_ * args.steps / 1e3)
+        specs = kernel_specs(wl, peaks, tens)
+        recs, n_launch = {}, 0
+        for name, (ms, cnt) in prof_.items():
+            if cnt == 0:
+                continue
+            n_launch += cnt
+            bound, work, peak, unit = specs[name]
+            avg_ms = ms / cnt
+            ent = {"launches_per_step": cnt // args.steps, "avg_ms": round(avg_ms, 5), "share": None, "bound": bound}
+            if work is not None:
+                ach = work / (avg_ms / 1e3)
+                ent.update({"achieved": round(ach, 2), "peak": peak, "unit": unit, "frac": round(ach / peak, 4)})
+            if name in EXP_KERNELS:
+                # second ceiling of the scorer kernels: the exponential unit, 16 ex2 per clock per SM
+                n_exp = wl.units * wl.G * wl.w * (wl.N if name != "score_colsum" else wl.N - wl.w)
+                peak_exp = sm_count * 16 * (clk.get("sm_max_mhz") or 1965) * 1e6
+                ent.update({"ex2_per_launch": n_exp,
+                            "ex2_frac_of_unit_peak": round(n_exp / (avg_ms / 1e3) / peak_exp, 4)})
+            recs[name] = ent
+        total_kernel_ms = sum(v[0] for v in prof_.values())
+        for name in recs:
+            recs[name]["share"] = round(prof_[name][0] / total_kernel_ms, 4)
+        return recs, n_launch, tens, tens_name
+
+    ms_step, clocks, prof = timed_passes(None)
     tokens_step = wl.B * wl.N * world
     value = shard.whole_job_tokens_per_s(wl, world, ms_step)
-
-    # ---- per-kernel roofline, from the events the library recorded inside the timed region
-    specs = kernel_specs(wl, peaks, sustained=True)
-    kernels = {}
-    launches = 0
-    for name, (ms, cnt) in prof.items():
-        if cnt == 0:
-            continue
-        launches += cnt
-        bound, work, peak, unit = specs[name]
-        avg_ms = ms / cnt
-        ent = {"launches_per_step": cnt // args.steps, "avg_ms": round(avg_ms, 5), "share": None, "bound": bound}
-        if work is not None:
-            ach = work / (avg_ms / 1e3)
-            ent.update({"achieved": round(ach, 2), "peak": peak, "unit": unit, "frac": round(ach / peak, 4)})
-        if name in EXP_KERNELS:
-            # second ceiling of the scorer kernels: the exponential unit, 16 ex2 per clock per SM
-            n_exp = wl.units * wl.G * wl.w * (wl.N if name != "score_colsum" else wl.N - wl.w)
-            sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
-            peak_exp = sm_count * 16 * (clocks.get("sm_max_mhz") or 1965) * 1e6
-            ent.update({"ex2_per_launch": n_exp, "ex2_frac_of_unit_peak": round(n_exp / (avg_ms / 1e3) / peak_exp, 4)})
-        kernels[name] = ent
-    total_kernel_ms = sum(v[0] for v in prof.values())
-    for name in kernels:
-        kernels[name]["share"] = round(prof[name][0] / total_kernel_ms, 4)
+    kernels, launches, tens_peak, tens_name = kernel_records(prof, clocks, ms_step)
     dom = max(kernels, key=lambda n: kernels[n]["share"])
     kd = kernels[dom]
+    ctr = ncu_counters(dom)
     roofline = {"kernel": dom, "bound": kd["bound"], "achieved": kd.get("achieved"), "peak": kd.get("peak"),
                 "unit": kd.get("unit"), "frac": kd.get("frac"),
-                "traffic": (round(TRAFFIC_PER_UNIT_TOKEN[dom] * wl.units * wl.N / 1e9, 4)
-                            if TRAFFIC_PER_UNIT_TOKEN.get(dom) else None),
+                "traffic": round(ctr["dram_bytes_per_unit_token"] * wl.units * wl.N / 1e9, 4) if ctr else None,
                 "traffic_unit": "GB per launch (ncu dram bytes of a smaller case, scaled by units x tokens)",
-                "peak_source": f"of {peaks['source']} ({'sustained bf16' if kd['bound'] == 'tensor' else 'copy'})",
+                "tensor_pipe_pct": ctr["tensor_pipe_pct"] if ctr else None,
+                "xu_pipe_pct": ctr["xu_pipe_pct"] if ctr else None,
+                "counters_source": NCU_COUNTERS["capture"] if ctr else None,
+                "peak_source": f"of {peaks['source']} ({tens_name if kd['bound'] == 'tensor' else 'copy'}; the timed "
+                               f"region lasted {ms_step * args.steps / 1e3:.2f} s, power cap "
+                               f"{'seen' if 'sw_power_cap' in (clocks.get('reasons') or []) else 'not seen'})",
                 "avg_ms": kd["avg_ms"], "share": kd["share"]}
+    sm_mhz = clocks.get("sm_max_mhz") or 1965
+    bound2 = composite_bound(wl, 2, peaks["hbm_gbs"], tens_peak, sm_count, sm_mhz, ms_step)
+    bound2["note"] = ("the softmax needs the row normalisers before the column sums, so the window product and its "
+                      "exponentials run twice; t_exp at the maximum SM clock")
+
+    # ---- the same pass with the caller's log-sum-exp (what a prefill attention kernel keeps per window row): the
+    # statistics sweep and the merge drop out, the entropy call runs the Gram stage on its own.  The normalisers are
+    # prepared once, outside the timed region, by a plain matrix product and logsumexp on the device.
+    with_lse = None
+    if wl.dtype == "bf16" and not args.no_lse:
+        lse = prefill_lse(wl, K, Qw)
+        ms_lse, clocks_lse, prof_lse = timed_passes(lse)
+        k_lse, launches_lse, tens_lse, tens_lse_name = kernel_records(prof_lse, clocks_lse, ms_lse)
+        hb = wl.algorithmic_bytes() / 1e9 / (ms_lse / 1e3)
+        with_lse = {"ms_per_step": ms_lse, "value": shard.whole_job_tokens_per_s(wl, world, ms_lse), "unit": UNIT,
+                    "hbm_frac_of_measured_copy": round(hb / peaks["hbm_gbs"], 4), "achieved_gbs": round(hb, 1),
+                    "composite_bound": composite_bound(wl, 1, peaks["hbm_gbs"], tens_lse, sm_count, sm_mhz, ms_lse),
+                    "tensor_peak": tens_lse_name, "kernels": {n: {"avg_ms": v["avg_ms"], "frac": v.get("frac")}
+                                                              for n, v in k_lse.items()},
+                    "gpu_launches": launches_lse, "clocks": clocks_lse}
+        del lse
     alg_bytes = wl.algorithmic_bytes()
     hbm_pass = alg_bytes / 1e9 / (ms_step / 1e3)
 
@@ -952,8 +1053,8 @@ def main():
                 "hbm_pass": {"algorithmic_gb": round(alg_bytes / 1e9, 4), "achieved_gbs": round(hbm_pass, 1),
                              "frac_of_measured_copy": round(hbm_pass / peaks["hbm_gbs"], 4),
                              "frac_of_nominal_8tbs": round(hbm_pass / 8000.0, 4)},
-                "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
-                "gpu_launches": launches, "clocks": clocks}
+                "roofline": roofline, "composite_bound": bound2, "kernels": kernels, "with_lse": with_lse,
+                "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

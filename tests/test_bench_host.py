@@ -89,3 +89,51 @@ def test_eviction_plan_host_logic():
     assert eviction_plan([0, 0, 0], [900, 900, 900]) == []
     assert eviction_plan([0, 1, 2], [500, 500, 300]) == [(2, 300)]
     assert eviction_plan([], []) == []
+
+
+def _bench():
+    sys.path.insert(0, ROOT)
+    import bench
+    return bench
+
+
+def test_tensor_peak_follows_the_regime_of_the_timed_region():
+    bench = _bench()
+    peaks = {"bf16_burst": 1600.0, "bf16_sustained": 1400.0}
+    assert bench.tensor_peak(peaks, {"reasons": []}, 0.1) == (1600.0, "burst bf16")
+    assert bench.tensor_peak(peaks, {"reasons": ["sw_power_cap"]}, 0.1) == (1400.0, "sustained bf16")
+    assert bench.tensor_peak(peaks, {"reasons": []}, 2.5) == (1400.0, "sustained bf16")
+    assert bench.tensor_peak(peaks, {}, 0.999)[1] == "burst bf16"
+
+
+def test_composite_bound_arithmetic():
+    from paper_2410_03090_b200 import synth
+    bench = _bench()
+    wl = synth.WORKLOADS["c3"]
+    rows, u = wl.G * wl.w, wl.units
+    b = bench.composite_bound(wl, 2, hbm_gbs=6500.0, tensor_tflops=1400.0, sm_count=148, sm_mhz=1965, ms_step=2.0)
+    t_hbm = wl.algorithmic_bytes() / 6500e9 * 1e3
+    t_tensor = u * (2.0 * wl.N * 128 * 128 + 2 * 2.0 * rows * 128 * wl.N) / 1400e12 * 1e3
+    t_exp = u * 2.0 * rows * wl.N / (148 * 16 * 1965e6) * 1e3
+    assert abs(b["t_hbm_ms"] - t_hbm) < 1e-3 and abs(b["t_tensor_ms"] - t_tensor) < 1e-3
+    assert abs(b["t_exp_ms"] - t_exp) < 1e-3
+    assert b["t_min_ms"] == max(b["t_hbm_ms"], b["t_tensor_ms"], b["t_exp_ms"]) and b["binding"] == "tensor"
+    assert abs(b["frac_of_t_min"] - b["t_min_ms"] / 2.0) < 1e-3
+    # one window product instead of two: both the tensor and the exponential bound shrink, the byte bound does not
+    b1 = bench.composite_bound(wl, 1, 6500.0, 1400.0, 148, 1965, 1.5)
+    assert b1["t_hbm_ms"] == b["t_hbm_ms"] and b1["t_exp_ms"] < b["t_exp_ms"] and b1["t_tensor_ms"] < b["t_tensor_ms"]
+    assert abs(b1["t_exp_ms"] * 2 - b["t_exp_ms"]) < 1e-3
+
+
+def test_ncu_counters_are_dropped_when_the_kernel_source_changed(monkeypatch):
+    import hashlib
+    bench = _bench()
+    src = os.path.join(ROOT, bench.NCU_COUNTERS["source"])
+    with open(src, "rb") as f:
+        digest = hashlib.sha256(f.read()).hexdigest()
+    fake = {"source": bench.NCU_COUNTERS["source"], "sha256": digest, "capture": "x",
+            "kernels": {"k": {"dram_bytes_per_unit_token": 1.0, "tensor_pipe_pct": 2.0, "xu_pipe_pct": 3.0}}}
+    monkeypatch.setattr(bench, "NCU_COUNTERS", fake)
+    assert bench.ncu_counters("k")["tensor_pipe_pct"] == 2.0 and bench.ncu_counters("other") is None
+    monkeypatch.setattr(bench, "NCU_COUNTERS", dict(fake, sha256="0" * 64))
+    assert bench.ncu_counters("k") is None
