@@ -194,7 +194,7 @@ __device__ __forceinline__ void householder_block(float (&A)[8][8], E32Smem &S, 
 #pragma unroll
         for (int a = KA; a < 8; ++a)
 #pragma unroll
-            for (int b = KA; b < 8; ++b) A[a][b] -= fmaf(vr[a], wc[b], wr[a] * vc[b]);
+            for (int b = KA; b < 8; ++b) A[a][b] = fmaf(-wr[a], vc[b], fmaf(-vr[a], wc[b], A[a][b]));
     }
 }
 }  // namespace
@@ -340,20 +340,26 @@ eigen_f32_kernel(const float *__restrict__ partials, int P, int N, int k_trunc, 
     __syncthreads();
 
     // ---- 4. entropy -----------------------------------------------------------------------------
-    if (tid == 0) {
+    if (wid == 0) {      // one warp: lane i takes eigenvalues i, i + 32, ...; fixed-order butterfly sums
         double total = 0.0;
         if (norm) total = trace > 0.0 ? 1.0 : 0.0;
-        else for (int i = 0; i < k; ++i) total += S.lam[i] > 0.0 ? S.lam[i] : 0.0;
+        else {
+            for (int i = lane; i < k; i += 32) total += S.lam[i] > 0.0 ? S.lam[i] : 0.0;
+            total = warp_sum(total);
+        }
         double h = 0.0;
         if (total > 0.0) {
-            for (int i = 0; i < k; ++i) {
+            for (int i = lane; i < k; i += 32) {
                 const double p = (S.lam[i] > 0.0 ? S.lam[i] : 0.0) / total;
                 if (p > 0.0) h -= p * log(p);
             }
         }
-        entropy[u] = (float)h;
-        if (erank) erank[u] = (float)exp(h);
-        if (S.flags[0]) atomicOr(status, (uint32_t)UNCOMP_STATUS_NOT_CONVERGED);
+        h = warp_sum(h);
+        if (lane == 0) {
+            entropy[u] = (float)h;
+            if (erank) erank[u] = (float)exp(h);
+            if (S.flags[0]) atomicOr(status, (uint32_t)UNCOMP_STATUS_NOT_CONVERGED);
+        }
     }
     if (spectrum && tid < k) spectrum[(size_t)u * k + tid] = S.lam[tid] * trace;
 }
