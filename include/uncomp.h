@@ -407,6 +407,22 @@ int uncomp_entropy_wide(uncomp_ctx *ctx, const void *d_X, int32_t count, int64_t
                         float *d_entropy, float *d_erank, double *d_spectrum, void *stream);
 
 /* ---------------------------------------------------------------------------------------------------
+ * uncomp_eviction_plan -- Section 3.3.2 "Hidden State Eviction"; Algorithm 2, "compress hidden states":
+ * where the prefill cuts the hidden states, read off the layer partition of ONE sequence as
+ * uncomp_assign_budgets writes it.  Host function on HOST arrays (copy the L entries of the sequence back
+ * first); launches nothing.  Before layer l, the first layer of a new layer group whose context is
+ * smaller than what is still there, the hidden states are cut to layer_ctx[l] positions
+ * (uncomp_evict_hidden with n_keep = layer_ctx[l], scored by layer l - 1).  A group whose context is not
+ * smaller needs no call and is left out.
+ *
+ * layer_group, layer_ctx  in   [L] int32, host
+ * out_layer, out_keep     out  [L] int32, host: the first `return value` entries are the calls to make
+ * Returns the number of entries, or a negative error code (UNCOMP_E_NULL, UNCOMP_E_PARAM for L < 0).
+ * ------------------------------------------------------------------------------------------------- */
+int uncomp_eviction_plan(const int32_t *layer_group, const int32_t *layer_ctx, int32_t L, int32_t *out_layer,
+                         int32_t *out_keep);
+
+/* ---------------------------------------------------------------------------------------------------
  * uncomp_retrieval_layer -- Section 3.3.2 "Retrieval Layer": the retrieval layer is chosen as the layer of
  * maximum entropy increase.  d_values [L, H] holds a per-head value (the truncated entropy or the
  * effective rank, of one input or averaged by uncomp_prepare_groups); with e_l its mean over the heads of

@@ -44,9 +44,11 @@ class uncomp_score_params(C.Structure):
 
 
 def _load() -> C.CDLL:
-    path = _build.LIB
+    # UNCOMP_DEBUG_LIBRARY=1 selects the bounds-checked build of the same sources (libuncomp_debug.so)
+    debug = os.environ.get("UNCOMP_DEBUG_LIBRARY") == "1"
+    path = _build.LIB_DEBUG if debug else _build.LIB
     if not os.path.exists(path):
-        path = _build.build()
+        path = _build.build(debug=debug)
     lib = C.CDLL(path)
     vp, i32p, i64p, fp, dp = C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p
     lib.uncomp_version.restype = C.c_int
@@ -88,6 +90,8 @@ def _load() -> C.CDLL:
     lib.uncomp_entropy_wide.restype = C.c_int
     lib.uncomp_entropy_wide.argtypes = [vp, vp, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
                                         C.POINTER(uncomp_entropy_params), vp, C.c_size_t, fp, fp, dp, vp]
+    lib.uncomp_eviction_plan.restype = C.c_int
+    lib.uncomp_eviction_plan.argtypes = [vp, vp, C.c_int32, vp, vp]
     lib.uncomp_retrieval_layer.restype = C.c_int
     lib.uncomp_retrieval_layer.argtypes = [vp, fp, i32p, fp, vp]
     lib.uncomp_prepare_groups.restype = C.c_int
@@ -242,6 +246,22 @@ def uncomp_score_select(ctx: Context, Qw: torch.Tensor, K: torch.Tensor, budgets
                                    _ptr(offsets), C.byref(p), _ptr(scores), _ptr(indices), _stream(stream)),
            "uncomp_score_select")
     return indices
+
+
+def uncomp_eviction_plan(layer_group, layer_ctx):
+    """Host rows [L] of one sequence (lists, numpy or CPU tensors) -> [(layer, n_keep)]."""
+    import numpy as np
+    g = np.ascontiguousarray(np.asarray(layer_group, dtype=np.int32).reshape(-1))
+    c = np.ascontiguousarray(np.asarray(layer_ctx, dtype=np.int32).reshape(-1))
+    if g.shape != c.shape:
+        raise ValueError("layer_group and layer_ctx must have the same length")
+    L = int(g.shape[0])
+    out_l, out_k = np.zeros(max(L, 1), dtype=np.int32), np.zeros(max(L, 1), dtype=np.int32)
+    n = lib.uncomp_eviction_plan(C.c_void_p(g.ctypes.data), C.c_void_p(c.ctypes.data), L,
+                                 C.c_void_p(out_l.ctypes.data), C.c_void_p(out_k.ctypes.data))
+    if n < 0:
+        raise UncompError(n, "uncomp_eviction_plan")
+    return [(int(out_l[i]), int(out_k[i])) for i in range(n)]
 
 
 def uncomp_compact(ctx: Context, K: torch.Tensor, V: torch.Tensor, indices: torch.Tensor, offsets: torch.Tensor,

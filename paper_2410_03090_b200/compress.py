@@ -80,19 +80,9 @@ class CompressionPass:
 
 
 def eviction_plan(layer_group, layer_ctx):
-    """Where the prefill evicts hidden states (paper Section 3.3.2; Algorithm 2, "compress hidden states"): host
-    logic over the `layer_group` / `layer_ctx` rows of one sequence as `uncomp_assign_budgets` writes them.
-    Returns [(layer, n_keep)]: before layer `layer` (the first of a new layer group) the hidden states are cut to
-    the `n_keep` positions with the highest last-token attention of layer `layer - 1` (`uncomp_evict_hidden`).
-    A group whose context is not smaller than what is still there needs no call and is left out."""
-    groups = [int(g) for g in layer_group]
-    ctx = [int(c) for c in layer_ctx]
-    plan, current = [], ctx[0] if ctx else 0
-    for l in range(1, len(groups)):
-        if groups[l] != groups[l - 1] and ctx[l] < current:
-            plan.append((l, ctx[l]))
-            current = ctx[l]
-    return plan
+    """[(layer, n_keep)] for one sequence: marshals the two host rows into `uncomp_eviction_plan` (the rule itself,
+    paper Section 3.3.2, lives in the library)."""
+    return ub.uncomp_eviction_plan(layer_group, layer_ctx)
 
 
 class DecodeCache:

@@ -431,6 +431,24 @@ int uncomp_decode_update(uncomp_ctx *ctx, const void *d_qnew, const void *d_knew
     return UNCOMP_OK;
 }
 
+int uncomp_eviction_plan(const int32_t *layer_group, const int32_t *layer_ctx, int32_t L, int32_t *out_layer,
+                         int32_t *out_keep) {
+    if (L < 0) return UNCOMP_E_PARAM;
+    if (L == 0) return 0;
+    if (!layer_group || !layer_ctx || !out_layer || !out_keep) return UNCOMP_E_NULL;
+    int n = 0;
+    int32_t current = layer_ctx[0];
+    for (int32_t l = 1; l < L; ++l) {
+        if (layer_group[l] != layer_group[l - 1] && layer_ctx[l] < current) {
+            out_layer[n] = l;
+            out_keep[n] = layer_ctx[l];
+            current = layer_ctx[l];
+            ++n;
+        }
+    }
+    return n;
+}
+
 int uncomp_retrieval_layer(uncomp_ctx *ctx, const float *d_values, int32_t *d_layer, float *d_increase, void *stream) {
     if (!ctx || !d_values || !d_layer) return UNCOMP_E_NULL;
     const uncomp_shape &s = ctx->plan.shape;

@@ -49,6 +49,21 @@ inline UnitAddr make_addr(const uncomp_shape &s, const uncomp_strides &st) {
     return a;
 }
 
+// Debug library (-DUNCOMP_DEBUG, built as libuncomp_debug.so): the kernels that place data at computed positions
+// (selection, compaction, decode-time commit, hidden-state gather) check every such
+// index against the extent it must stay in.  A violation raises UNCOMP_STATUS_BOUNDS and the access is skipped:
+// no trap, no assert.  In the release library the check is the constant `true`.
+#ifdef UNCOMP_DEBUG
+__device__ __forceinline__ bool debug_index_ok(int64_t i, int64_t extent, uint32_t *status) {
+    if (i >= 0 && i < extent) return true;
+    atomicOr(status, (uint32_t)UNCOMP_STATUS_BOUNDS);
+    return false;
+}
+#define UNCOMP_INDEX_OK(i, extent, status) (::uncomp::debug_index_ok((int64_t)(i), (int64_t)(extent), (status)))
+#else
+#define UNCOMP_INDEX_OK(i, extent, status) (true)
+#endif
+
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 

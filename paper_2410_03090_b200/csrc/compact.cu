@@ -36,6 +36,7 @@ __global__ void __launch_bounds__(256) compact_kernel(const unsigned char *__res
                 const int mid = (lo + hi + 1) >> 1;
                 if (offsets[mid] <= t) lo = mid; else hi = mid - 1;
             }
+            if (!UNCOMP_INDEX_OK(lo, units, status)) lo = 0;
             int64_t idx = indices[t];
             if (idx < 0 || idx >= N) {        // never form an address outside the unit's rows
                 atomicOr(status, (uint32_t)UNCOMP_STATUS_BOUNDS);
@@ -50,7 +51,7 @@ __global__ void __launch_bounds__(256) compact_kernel(const unsigned char *__res
             const int row = r + sub;
             const int64_t sk = __shfl_sync(0xffffffffu, srcK, row);
             const int64_t sv = __shfl_sync(0xffffffffu, srcV, row);
-            if (row < nrows) {
+            if (row < nrows && UNCOMP_INDEX_OK(t0 + row, total, status)) {
                 const int4 a = *reinterpret_cast<const int4 *>(K + sk + vec * 16);
                 const int4 b = *reinterpret_cast<const int4 *>(V + sv + vec * 16);
                 const int64_t dst = (t0 + row) * ROW_BYTES + vec * 16;

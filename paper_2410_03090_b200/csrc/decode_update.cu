@@ -328,13 +328,17 @@ __global__ void __launch_bounds__(64) decode_commit_kernel(DecArgs a, int H_per_
         } else {
             lens[u] = len + 1;
         }
-        pos[off + slot] = new_pos[u / H_per_seq];
-        cum[off + slot] = new_cum[u];
+        if (!UNCOMP_INDEX_OK(slot, cap, status)) slot = -1;       // debug library: the row must lie in the unit's slab
+        if (slot >= 0) {
+            pos[off + slot] = new_pos[u / H_per_seq];
+            cum[off + slot] = new_cum[u];
+        }
         if (evicted) evicted[u] = gone;
         slot_s = slot;
     }
     __syncthreads();
     const int slot = slot_s, vecs = row_bytes >> 4;      // 16-byte vectors per row: 16 (bf16) or 32 (fp32)
+    if (slot < 0) return;                                // only the debug library can get here
     const int4 *srcK = reinterpret_cast<const int4 *>((const char *)a.knew + (size_t)u * row_bytes);
     const int4 *srcV = reinterpret_cast<const int4 *>((const char *)vnew + (size_t)u * row_bytes);
     int4 *dstK = reinterpret_cast<int4 *>((char *)Kc + (off + slot) * row_bytes);

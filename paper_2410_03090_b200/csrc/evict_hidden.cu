@@ -289,12 +289,14 @@ __global__ void __launch_bounds__(kEvThreads) last_token_scores_kernel(
 // one warp per kept row: Xout[b, t, :] = X[b, idx[b, t], :]
 __global__ void __launch_bounds__(256) gather_rows_kernel(const unsigned char *__restrict__ X,
                                                          const int32_t *__restrict__ idx, int64_t rows_total, int n_keep,
-                                                         int N, int64_t row_bytes, unsigned char *__restrict__ out) {
+                                                         int N, int64_t row_bytes, unsigned char *__restrict__ out,
+                                                         uint32_t *__restrict__ status) {
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     for (int64_t t = warp; t < rows_total; t += nwarps) {
         const int64_t b = t / n_keep;
+        if (!UNCOMP_INDEX_OK(idx[t], N, status)) continue;
         const int4 *src = reinterpret_cast<const int4 *>(X + (b * N + idx[t]) * row_bytes);
         int4 *dst = reinterpret_cast<int4 *>(out + t * row_bytes);
         const int nvec = (int)(row_bytes >> 4);
@@ -374,7 +376,7 @@ cudaError_t launch_evict_hidden(const Plan &p, const void *d_qlast, const void *
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         gather_rows_kernel<<<sms * 8, 256, 0, st>>>((const unsigned char *)d_X, d_indices, (int64_t)s.B * n_keep, n_keep,
-                                                    s.N, row_bytes, (unsigned char *)d_Xout);
+                                                    s.N, row_bytes, (unsigned char *)d_Xout, d_status);
     }
     return cudaGetLastError();
 }

@@ -38,7 +38,7 @@ struct SelSmem {
 // slab and the budget both allow, so that every slot of the slab holds a valid position and nothing outside it
 // is touched: k top positions, then wn window positions, then `fill` copies of the last position.
 struct Slab {
-    int64_t begin;
+    int64_t begin, seg;
     int k, wn;
     int64_t fill;
 };
@@ -55,6 +55,7 @@ __device__ __forceinline__ Slab slab_of(const int32_t *__restrict__ budgets, con
     b = min(b, seg);
     Slab s;
     s.begin = off_ok ? o0 : 0;
+    s.seg = seg;
     s.k = (int)max((int64_t)0, min(b - w, (int64_t)P));
     s.wn = (int)min((int64_t)w, b - s.k);
     s.fill = seg - s.k - s.wn;
@@ -104,8 +105,10 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float *_
     const Slab slab = slab_of(budgets, offsets, units, u, P, w, tid == 0, status);
     const int k = slab.k;
     int32_t *out = indices + slab.begin;
-    for (int i = tid; i < slab.wn; i += kSelThreads) out[k + i] = P + i;
-    for (int64_t i = tid; i < slab.fill; i += kSelThreads) out[k + slab.wn + i] = P + w - 1;
+    for (int i = tid; i < slab.wn; i += kSelThreads)
+            if (UNCOMP_INDEX_OK(k + i, slab.seg, status)) out[k + i] = P + i;
+    for (int64_t i = tid; i < slab.fill; i += kSelThreads)
+            if (UNCOMP_INDEX_OK(k + slab.wn + i, slab.seg, status)) out[k + slab.wn + i] = P + w - 1;
     if (k == 0) return;   // uniform over the CTA
     __syncthreads();      // pooled scores of this unit are visible to the whole CTA
 
@@ -123,7 +126,8 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float *_
             __syncthreads();
             for (int j = tid; j < P; j += kSelThreads) {
                 const uint32_t v = ordered_bits(s[j]);
-                if ((v & himask) == prefix) atomicAdd(&S.hist[(v >> shift) & (nbins - 1)], 1);
+                if ((v & himask) == prefix && UNCOMP_INDEX_OK((v >> shift) & (nbins - 1), 2048, status))
+                    atomicAdd(&S.hist[(v >> shift) & (nbins - 1)], 1);
             }
             __syncthreads();
             find_bin(S, nbins, kr, tid);
@@ -163,7 +167,8 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const float *_
         const unsigned mg = __ballot_sync(0xffffffffu, gt), me = __ballot_sync(0xffffffffu, eq);
         const int gtb = gt_run + __popc(mg & lt);
         const int eqb = eq_run + __popc(me & lt);
-        if (gt || (eq && eqb < need_eq)) out[gtb + min(eqb, need_eq)] = j;
+        if ((gt || (eq && eqb < need_eq)) && UNCOMP_INDEX_OK(gtb + min(eqb, need_eq), k, status))
+            out[gtb + min(eqb, need_eq)] = j;
         gt_run += __popc(mg);
         eq_run += __popc(me);
     }
@@ -202,8 +207,10 @@ pool_select_cluster_kernel(const float *__restrict__ raw, float *__restrict__ po
     const int k = slab.k;
     int32_t *out = indices + slab.begin;
     if (rank == 0) {
-        for (int i = tid; i < slab.wn; i += kSelThreads) out[k + i] = P + i;
-        for (int64_t i = tid; i < slab.fill; i += kSelThreads) out[k + slab.wn + i] = P + w - 1;
+        for (int i = tid; i < slab.wn; i += kSelThreads)
+            if (UNCOMP_INDEX_OK(k + i, slab.seg, status)) out[k + i] = P + i;
+        for (int64_t i = tid; i < slab.fill; i += kSelThreads)
+            if (UNCOMP_INDEX_OK(k + slab.wn + i, slab.seg, status)) out[k + slab.wn + i] = P + w - 1;
     }
     if (k == 0) return;   // uniform over the cluster
     __syncthreads();      // this CTA reads only the pooled scores it wrote itself
@@ -222,7 +229,8 @@ pool_select_cluster_kernel(const float *__restrict__ raw, float *__restrict__ po
             __syncthreads();
             for (int j = p0 + tid; j < p1; j += kSelThreads) {
                 const uint32_t v = ordered_bits(s[j]);
-                if ((v & himask) == prefix) atomicAdd(&S.hist[(v >> shift) & (nbins - 1)], 1);
+                if ((v & himask) == prefix && UNCOMP_INDEX_OK((v >> shift) & (nbins - 1), 2048, status))
+                    atomicAdd(&S.hist[(v >> shift) & (nbins - 1)], 1);
             }
             cluster.sync();                       // every CTA's histogram is complete
             if (rank == 0) {
@@ -281,7 +289,8 @@ pool_select_cluster_kernel(const float *__restrict__ raw, float *__restrict__ po
         const unsigned mg = __ballot_sync(0xffffffffu, gt), me = __ballot_sync(0xffffffffu, eq);
         const int gtb = gt_run + __popc(mg & lt);
         const int eqb = eq_run + __popc(me & lt);
-        if (gt || (eq && eqb < need_eq)) out[gtb + min(eqb, need_eq)] = j;
+        if ((gt || (eq && eqb < need_eq)) && UNCOMP_INDEX_OK(gtb + min(eqb, need_eq), k, status))
+            out[gtb + min(eqb, need_eq)] = j;
         gt_run += __popc(mg);
         eq_run += __popc(me);
     }
