@@ -31,9 +31,14 @@ if ROOT not in sys.path:
 # recorded beside them: when the file has changed since the capture, the bench prints null instead.
 NCU_COUNTERS = {
     "source": "paper_2410_03090_b200/csrc/scores_tc.cu",
-    "sha256": "",
-    "capture": "",
-    "kernels": {},
+    "sha256": "956983e80c73a67a6cf70cf9cae8510b9b85f474274958c13cbb7b3a01550ae8",
+    "capture": "ncu --set full, one launch per kernel, c3 scaled to N 16384 x 10 layers; summary in profiles/",
+    "kernels": {
+        "gram_score_stats": {"dram_bytes_per_unit_token": (342.103040e6 + 22.506752e6) / (80 * 16384),
+                             "tensor_pipe_pct": 39.8, "xu_pipe_pct": 54.2},
+        "score_colsum": {"dram_bytes_per_unit_token": (340.977664e6 + 7.157248e6) / (80 * 16384),
+                         "tensor_pipe_pct": 36.2, "xu_pipe_pct": 72.4},
+    },
 }
 EXP_KERNELS = ("score_stats", "score_colsum", "gram_score_stats")
 METRIC = "compression_pass_tokens_per_s"
