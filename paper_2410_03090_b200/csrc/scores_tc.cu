@@ -129,12 +129,23 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                 const float *__restrict__ mprime, float *__restrict__ raw, float *__restrict__ gram_part,
                 const void *__restrict__ Kraw, const UnitAddr kaddr, uint32_t *__restrict__ status) {
     constexpr bool PASS_B = MODE == 1, GRAM = MODE == 2;
-    constexpr int NB = GRAM ? 3 : kNB;               // accumulator ring: item n lives in buffer n % NB
-    // "Item n is ready" is signalled on barrier n % (2 NB): a softmax group that waits for the first item of its
-    // next tile may get there before the other group's item n - NB has completed, and with one barrier per buffer
-    // the parity of that unfinished phase could not be told from the one waited for.  The user of this barrier
-    // before item n is item n - 2 NB, which lies in a tile this group has already consumed (2 NB > MB).
+    // Accumulator buffers (128 TMEM columns each).  An item is one 128-row block of one tile; tile i belongs to
+    // softmax group i & 1.  Modes 0 and 1: four buffers, two owned by each group, which it fills alternately
+    // with its own items (so each group runs up to two items ahead, independent of the other).  Mode 2: the
+    // Gram block leaves room for three, which form one ring over all items in issue order.
+    constexpr int NB = GRAM ? 3 : kNB;
+    // Mode 2: "item n is ready" is signalled on barrier n % (2 NB).  A softmax group that waits for the first item
+    // of its next tile may get there before the other group's item n - NB has completed, and with one barrier per
+    // buffer the parity of that unfinished phase could not be told from the one waited for.  The user of barrier
+    // n % (2 NB) before item n is item n - 2 NB, which lies in a tile this group has already consumed (2 NB > MB).
+    // Modes 0 and 1 need no such care: a group only ever waits on its own buffers.
     constexpr int NF = 2 * NB;
+    // item (tile i, block mb) -> buffer, ready barrier and its parity, and the drain phase the MMA thread waits for
+    // (-1: the buffer has not been used yet)
+    auto item_buf = [](int i, int mb) { return GRAM ? (i * MB + mb) % NB : 2 * (i & 1) + (((i >> 1) * MB + mb) & 1); };
+    auto item_ready_bar = [](int i, int mb) { return GRAM ? (i * MB + mb) % NF : 2 * (i & 1) + (((i >> 1) * MB + mb) & 1); };
+    auto item_ready_parity = [](int i, int mb) { return GRAM ? ((i * MB + mb) / NF) & 1 : ((((i >> 1) * MB + mb) >> 1) & 1); };
+    auto item_drain_phase = [](int i, int mb) { return GRAM ? (i * MB + mb) / NB - 1 : ((((i >> 1) * MB + mb) >> 1) - 1); };
     constexpr uint32_t kGramCol = 384;               // TMEM columns of the Gram block (mode 2)
     constexpr int S = score_stages(MB);
     extern __shared__ unsigned char smem_raw[];
@@ -247,11 +258,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                 const uint32_t k_lo = k_lo0 + (uint32_t)(s * (kBlockBytes >> 4));
 #pragma unroll
                 for (int mb = 0; mb < MB; ++mb) {
-                    // item n (tile i, row block mb) goes to ring buffer n % NB, once item n - NB has been drained
-                    const int n = i * MB + mb, buf = n % NB;
-                    if (ok && n >= NB) {
+                    // the item's buffer must have been drained of its previous item
+                    const int buf = item_buf(i, mb), drain = item_drain_phase(i, mb);
+                    if (ok && drain >= 0) {
                         const uint32_t bar = tc::smem_u32(&T.tempty[buf]);
-                        const uint32_t parity = ((n / NB) - 1) & 1;
+                        const uint32_t parity = drain & 1;
                         if (GRAM) {
                             uint32_t spins = 0;
                             while (!tc::mbar_try_wait(bar, parity)) {
@@ -275,7 +286,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                         if (PASS_B) tc::mma_f16_ss_lohi(d_tmem, k_lo + off, q_lo[mb] + off, dhi, idesc, k > 0);
                         else tc::mma_f16_ss_lohi(d_tmem, q_lo[mb] + off, k_lo + off, dhi, idesc, k > 0);
                     }
-                    tc::mma_commit(tc::smem_u32(&T.tfull[n % NF]));
+                    tc::mma_commit(tc::smem_u32(&T.tfull[item_ready_bar(i, mb)]));
                 }
                 if (!ok) break;
                 if (GRAM) {
@@ -346,10 +357,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
             float acc = 0.f;
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
-                const int n = i * MB + mb, buf = n % NB;
+                const int buf = item_buf(i, mb);
                 uint32_t v[64];
                 if (!dead) {
-                    const bool ok = tc::mbar_wait(tc::smem_u32(&T.tfull[n % NF]), (n / NF) & 1, status);
+                    const bool ok = tc::mbar_wait(tc::smem_u32(&T.tfull[item_ready_bar(i, mb)]), item_ready_parity(i, mb),
+                                                  status);
                     dead = !__all_sync(0xffffffffu, ok);
                 }
                 if (!dead) {
