@@ -406,6 +406,13 @@ int uncomp_entropy_wide(uncomp_ctx *ctx, const void *d_X, int32_t count, int64_t
                         int32_t N, int32_t D, const uncomp_entropy_params *params, void *d_scratch, size_t scratch_bytes,
                         float *d_entropy, float *d_erank, double *d_spectrum, void *stream);
 
+/* uncomp_measure_l2_sweep -- measurement aid, no counterpart in the paper: the memory pattern of the
+ * tridiagonalisation sweep of uncomp_entropy_wide on its own (a warp per row, every element read, changed by
+ * one fused multiply-add and written back, `passes` times).  Timed by the caller with events on `stream`, a
+ * matrix that fits in L2 gives the bandwidth that sweep can be held against.  d_A [rows, cols] float, device,
+ * 16-byte aligned, cols a multiple of 4; its contents are overwritten. */
+int uncomp_measure_l2_sweep(float *d_A, int32_t rows, int32_t cols, int32_t passes, void *stream);
+
 /* ---------------------------------------------------------------------------------------------------
  * uncomp_eviction_plan -- Section 3.3.2 "Hidden State Eviction"; Algorithm 2, "compress hidden states":
  * where the prefill cuts the hidden states, read off the layer partition of ONE sequence as

@@ -90,6 +90,8 @@ def _load() -> C.CDLL:
     lib.uncomp_entropy_wide.restype = C.c_int
     lib.uncomp_entropy_wide.argtypes = [vp, vp, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
                                         C.POINTER(uncomp_entropy_params), vp, C.c_size_t, fp, fp, dp, vp]
+    lib.uncomp_measure_l2_sweep.restype = C.c_int
+    lib.uncomp_measure_l2_sweep.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, vp]
     lib.uncomp_eviction_plan.restype = C.c_int
     lib.uncomp_eviction_plan.argtypes = [vp, vp, C.c_int32, vp, vp]
     lib.uncomp_retrieval_layer.restype = C.c_int
@@ -246,6 +248,14 @@ def uncomp_score_select(ctx: Context, Qw: torch.Tensor, K: torch.Tensor, budgets
                                    _ptr(offsets), C.byref(p), _ptr(scores), _ptr(indices), _stream(stream)),
            "uncomp_score_select")
     return indices
+
+
+def uncomp_measure_l2_sweep(A: torch.Tensor, passes: int = 1, stream=None) -> None:
+    """A [rows, cols] float32 on the device (overwritten): `passes` read-modify-write sweeps, for timing."""
+    if A.dtype != torch.float32 or A.dim() != 2 or not A.is_contiguous():
+        raise ValueError("expected a contiguous float32 matrix")
+    _check(lib.uncomp_measure_l2_sweep(_ptr(A), A.shape[0], A.shape[1], passes, _stream(stream)),
+           "uncomp_measure_l2_sweep")
 
 
 def uncomp_eviction_plan(layer_group, layer_ctx):

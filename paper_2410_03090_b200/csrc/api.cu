@@ -504,6 +504,14 @@ int uncomp_entropy_wide(uncomp_ctx *ctx, const void *d_X, int32_t count, int64_t
     return UNCOMP_OK;
 }
 
+int uncomp_measure_l2_sweep(float *d_A, int32_t rows, int32_t cols, int32_t passes, void *stream) {
+    if (!d_A) return UNCOMP_E_NULL;
+    if (rows < 1 || cols < 4 || cols % 4 != 0 || passes < 1) return UNCOMP_E_PARAM;
+    if (!aligned16(d_A)) return UNCOMP_E_ALIGN;
+    return launch_l2_sweep(d_A, rows, cols, passes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? UNCOMP_OK
+                                                                                                       : UNCOMP_E_CUDA;
+}
+
 int uncomp_evict_hidden(uncomp_ctx *ctx, const void *d_qlast, const void *d_K, uncomp_strides sK, const void *d_X,
                         int32_t D, int32_t n_keep, float scale, float *d_scores, int32_t *d_indices, void *d_Xout,
                         void *stream) {

@@ -148,6 +148,7 @@ size_t entropy_wide_scratch_bytes(int N, int D);
 cudaError_t launch_entropy_wide(const void *d_X, int64_t sN, int N, int D, const uncomp_entropy_params &ep,
                                 unsigned char *scratch, float *d_entropy, float *d_erank, double *d_spectrum,
                                 uint32_t *d_status, Profiler *prof, cudaStream_t st);
+cudaError_t launch_l2_sweep(float *d_A, int rows, int cols, int passes, cudaStream_t st);
 cudaError_t launch_compact(const Plan &p, const void *dK, const void *dV, const UnitAddr &aK, const UnitAddr &aV,
                            const int32_t *d_indices, const int64_t *d_offsets, void *dKc, void *dVc,
                            uint32_t *d_status, cudaStream_t st);

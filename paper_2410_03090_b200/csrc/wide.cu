@@ -466,6 +466,35 @@ __global__ void __launch_bounds__(kTriThreads, 1) tridiag_wide_kernel(float *__r
     }
 }
 
+// Measurement aid: the memory pattern of the sweep above on its own, so that the tridiagonalisation can be held
+// against a bandwidth measured on the same GPU.  A matrix of rows x cols floats that fits in L2 is read and written
+// once per pass, a warp per row, four 16-byte loads in flight per lane, one fused multiply-add per element.
+__global__ void __launch_bounds__(kTriThreads, 1) l2_sweep_kernel(float *__restrict__ A, int rows, int cols, int passes) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int total_warps = gridDim.x * kTriWarps, gw = warp * gridDim.x + blockIdx.x;
+    for (int p = 0; p < passes; ++p) {
+        for (int i = gw; i < rows; i += total_warps) {
+            float *row = A + (size_t)i * cols;
+            for (int jb = 4 * lane; jb < cols; jb += 512) {
+                float4 x[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    x[u] = jb + u * 128 < cols ? __ldcg(reinterpret_cast<const float4 *>(row + jb + u * 128))
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (jb + u * 128 < cols) {
+                        float4 y = x[u];
+                        y.x = fmaf(y.x, 0.999f, 1e-6f); y.y = fmaf(y.y, 0.999f, 1e-6f);
+                        y.z = fmaf(y.z, 0.999f, 1e-6f); y.w = fmaf(y.w, 0.999f, 1e-6f);
+                        __stcg(reinterpret_cast<float4 *>(row + jb + u * 128), y);
+                    }
+                }
+            }
+        }
+    }
+}
+
 // --------------------------------------------------------------------------------- 5. eigenvalues, entropy
 constexpr int kSturmThreads = 256;
 constexpr int kSturmMaxK = 256;
@@ -612,6 +641,16 @@ WideLayout wide_layout(int N, int D) {
     return w;
 }
 }  // namespace
+
+cudaError_t launch_l2_sweep(float *d_A, int rows, int cols, int passes, cudaStream_t st) {
+    int dev = 0, sms = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (err != cudaSuccess) return err;
+    l2_sweep_kernel<<<sms, kTriThreads, 0, st>>>(d_A, rows, cols, passes);
+    return cudaGetLastError();
+}
 
 size_t entropy_wide_scratch_bytes(int N, int D) { return wide_layout(N, D).bytes; }
 
