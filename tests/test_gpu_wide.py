@@ -97,3 +97,22 @@ def test_entropy_wide_rejections():
     with pytest.raises(ub.UncompError) as ei:
         ub.uncomp_entropy_wide(f32, X, 8)
     assert ei.value.code == ub.UNCOMP_E_SHAPE
+
+
+def test_l2_sweep_measurement_kernel_touches_every_element_once_per_pass():
+    """`uncomp_measure_l2_sweep` defines the denominator of the tridiagonalisation's roofline: one fused multiply-add
+    per element and pass, rows and ragged widths included, nothing outside the matrix."""
+    from paper_2410_03090_b200 import binding as ub
+    rows, cols, passes = 301, 4 * 131, 3
+    buf = torch.full((rows + 2, cols), 7.0, device="cuda")
+    A = buf[1:rows + 1]
+    A.copy_(torch.arange(rows * cols, device="cuda", dtype=torch.float32).reshape(rows, cols) / (rows * cols))
+    ref = A.clone().double()
+    ub.uncomp_measure_l2_sweep(A, passes)
+    torch.cuda.synchronize()
+    for _ in range(passes):
+        ref = ref * float(np.float32(0.999)) + float(np.float32(1e-6))
+    assert float((A.double() - ref).abs().max()) < 1e-6
+    assert float(buf[0].min()) == 7.0 and float(buf[-1].max()) == 7.0
+    with pytest.raises(ub.UncompError):
+        ub.uncomp_measure_l2_sweep(torch.zeros(4, 6, device="cuda"), 1)          # cols not a multiple of 4
