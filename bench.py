@@ -31,13 +31,13 @@ if ROOT not in sys.path:
 # recorded beside them: when the file has changed since the capture, the bench prints null instead.
 NCU_COUNTERS = {
     "source": "paper_2410_03090_b200/csrc/scores_tc.cu",
-    "sha256": "956983e80c73a67a6cf70cf9cae8510b9b85f474274958c13cbb7b3a01550ae8",
+    "sha256": "95d4b118eeb6fcb35f3939bddd07669b1930bca35ef0b6c8556135f72cdc081f",
     "capture": "ncu --set full, one launch per kernel, c3 scaled to N 16384 x 10 layers; summary in profiles/",
     "kernels": {
-        "gram_score_stats": {"dram_bytes_per_unit_token": (342.103040e6 + 22.506752e6) / (80 * 16384),
-                             "tensor_pipe_pct": 39.8, "xu_pipe_pct": 54.2},
-        "score_colsum": {"dram_bytes_per_unit_token": (340.977664e6 + 7.157248e6) / (80 * 16384),
-                         "tensor_pipe_pct": 36.2, "xu_pipe_pct": 72.4},
+        "gram_score_stats": {"dram_bytes_per_unit_token": (342.071552e6 + 25.281792e6) / (80 * 16384),
+                             "tensor_pipe_pct": 39.7, "xu_pipe_pct": 54.0},
+        "score_colsum": {"dram_bytes_per_unit_token": (340.974080e6 + 7.803136e6) / (80 * 16384),
+                         "tensor_pipe_pct": 35.8, "xu_pipe_pct": 71.5},
     },
 }
 EXP_KERNELS = ("score_stats", "score_colsum", "gram_score_stats")
