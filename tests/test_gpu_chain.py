@@ -20,10 +20,24 @@ import oracle
 import parity
 from paper_2410_03090_b200 import synth
 
-pytestmark = pytest.mark.gpu
 
 ERANK_GAP = 2e-4
 SCORE_GAP = 2e-3
+
+
+def _kept_position_diffs(got, ref, pooled, budget, w, where):
+    """Number of kept prefix positions in which `got` differs from the oracle's selection `ref`; raises unless every
+    differing position has an oracle score within SCORE_GAP (relative) of the oracle's k-th largest score."""
+    assert len(got) == len(ref) == budget, where
+    assert np.array_equal(got[-w:], ref[-w:]), where          # the window itself never differs
+    k = budget - w
+    if k == 0 or np.array_equal(got, ref):
+        return 0
+    odd = np.setxor1d(got[:k], ref[:k])
+    kth = np.sort(pooled)[::-1][k - 1]
+    rel = np.abs(pooled[odd] - kth) / kth
+    assert rel.max() < SCORE_GAP, f"{where}: position {odd[rel.argmax()]} differs, score gap {rel.max():.2e}"
+    return len(odd) // 2
 
 
 def _oracle_chain(wl, K, Qw):
@@ -37,7 +51,9 @@ def _oracle_chain(wl, K, Qw):
     return erank, bud, off, pooled
 
 
-@pytest.mark.parametrize("name,N,L,B", [("c2", 2048, 4, 1), ("c3", 4096, 2, 1), ("c4", 2048, 2, 2)])
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,N,L,B", [("c2", 2048, 4, 1), ("c3", 4096, 2, 1), ("c4", 2048, 2, 2),
+                                        ("c2", 8192, 32, 1)])          # the last one is workload c2 at its full size
 def test_whole_chain_differs_from_the_oracle_chain_only_at_near_ties(name, N, L, B):
     from paper_2410_03090_b200.compress import CompressionPass
     wl = synth.scaled(synth.WORKLOADS[name], N=N, L=L, B=B)
@@ -69,17 +85,24 @@ def test_whole_chain_differs_from_the_oracle_chain_only_at_near_ties(name, N, L,
         b, l, h = synth.unit_index(wl, u)
         budget = int(bud_g[b, l, h])
         ref = oracle.select(pooled_o[u], wl.w, budget)
-        got = idx_g[off_g[u]:off_g[u + 1]]
-        assert len(got) == len(ref) == budget
-        assert np.array_equal(got[-wl.w:], ref[-wl.w:])          # the window itself never differs
-        k = budget - wl.w
-        if k == 0 or np.array_equal(got, ref):
-            continue
-        odd = np.setxor1d(got[:k], ref[:k])
-        kth = np.sort(pooled_o[u])[::-1][k - 1]
-        rel = np.abs(pooled_o[u][odd] - kth) / kth
-        assert rel.max() < SCORE_GAP, f"unit {u}: position {odd[rel.argmax()]} differs, score gap {rel.max():.2e}"
-        index_diffs += len(odd) // 2
-        units_with_diffs += 1
+        n = _kept_position_diffs(idx_g[off_g[u]:off_g[u + 1]], ref, pooled_o[u], budget, wl.w, f"unit {u}")
+        index_diffs += n
+        units_with_diffs += n > 0
     print(f"\nchain mode {wl.name} ({wl.units} units, {int(off_g[-1])} kept rows): {budget_swaps} units with a swapped "
           f"budget, {index_diffs} differing kept positions in {units_with_diffs} units; all at near-ties")
+
+
+def test_the_position_check_itself_counts_near_ties_and_rejects_real_differences():
+    # CPU only: the checker above on hand-made selections.  Scores 10, 9, ..., with two near-equal ones at the cut.
+    pooled = np.array([10.0, 9.0, 8.0, 7.0, 6.0, 5.0 * (1 + 1e-4), 5.0, 4.0, 3.0, 2.0])
+    w, budget = 2, 8                                  # k = 6 kept prefix positions, then the window 10, 11
+    ref = oracle.select(pooled, w, budget)
+    assert ref.tolist() == [0, 1, 2, 3, 4, 5, 10, 11]
+    assert _kept_position_diffs(ref.copy(), ref, pooled, budget, w, "same") == 0
+    near = np.array([0, 1, 2, 3, 4, 6, 10, 11])       # takes position 6 instead of 5: scores 1e-4 apart
+    assert _kept_position_diffs(near, ref, pooled, budget, w, "near tie") == 1
+    far = np.array([0, 1, 2, 3, 4, 8, 10, 11])        # takes position 8 (score 3) instead of 5
+    with pytest.raises(AssertionError):
+        _kept_position_diffs(far, ref, pooled, budget, w, "real difference")
+    with pytest.raises(AssertionError):
+        _kept_position_diffs(np.array([0, 1, 2, 3, 4, 5, 9, 11]), ref, pooled, budget, w, "window touched")
