@@ -40,7 +40,7 @@ NCU_COUNTERS = {
                          "tensor_pipe_pct": 35.8, "xu_pipe_pct": 71.5},
     },
 }
-EXP_KERNELS = ("score_stats", "score_colsum", "gram_score_stats")
+EXP_KERNELS = ("score_stats", "score_colsum", "gram_score_stats", "gram_score_colsum")
 METRIC = "compression_pass_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -170,6 +170,7 @@ def kernel_specs(wl, peaks, sustained, D=None, n_keep=None, cache_rows=None):
     return {
         "gram": ("tensor", 2.0 * N * d * d * u / 1e12, tens, "TFLOP/s"),
         "gram_score_stats": ("tensor", (2.0 * N * d * d + 2.0 * rows * d * N) * u / 1e12, tens, "TFLOP/s"),
+        "gram_score_colsum": ("tensor", (2.0 * N * d * d + 2.0 * rows * d * N) * u / 1e12, tens, "TFLOP/s"),
         "score_stats": ("tensor", 2.0 * rows * d * N * u / 1e12, tens, "TFLOP/s"),
         "score_colsum": ("tensor", 2.0 * rows * d * P * u / 1e12, tens, "TFLOP/s"),
         "pool_select": ("hbm", (2.0 * u * P * 4 + wl.total_rows * 4) / 1e9, hbm, "GB/s"),
@@ -890,9 +891,11 @@ def main():
 
     def timed_passes(lse):
         """W warm-up and K timed passes (barrier + synchronize on both sides, CUDA events on the launching stream,
-        max over ranks); returns the step time, the clock record and the per-kernel event times."""
+        max over ranks); returns the step time, the clock record and the per-kernel event times.  Without
+        normalisers a pass is the four staged calls; with them it is the one-call form, which sweeps K once."""
+        run = cp.run if lse is None else cp.run_one_call
         for _ in range(args.warmup):
-            cp.run(K, V, Qw, lse=lse)
+            run(K, V, Qw, lse=lse)
         torch.cuda.synchronize()
         assert cp.status() == 0
         sampler = ClockSampler(local)
@@ -903,7 +906,7 @@ def main():
         torch.cuda.synchronize()
         ev0.record(stream)
         for _ in range(args.steps):
-            cp.run(K, V, Qw, lse=lse)
+            run(K, V, Qw, lse=lse)
         ev1.record(stream)
         torch.cuda.synchronize()
         barrier()
@@ -930,7 +933,7 @@ def main():
                 ent.update({"achieved": round(ach, 2), "peak": peak, "unit": unit, "frac": round(ach / peak, 4)})
             if name in EXP_KERNELS:
                 # second ceiling of the scorer kernels: the exponential unit, 16 ex2 per clock per SM
-                n_exp = wl.units * wl.G * wl.w * (wl.N if name != "score_colsum" else wl.N - wl.w)
+                n_exp = wl.units * wl.G * wl.w * (wl.N if name != "score_colsum" else wl.N - wl.w)   # tokens swept
                 peak_exp = sm_count * 16 * (clk.get("sm_max_mhz") or 1965) * 1e6
                 ent.update({"ex2_per_launch": n_exp,
                             "ex2_frac_of_unit_peak": round(n_exp / (avg_ms / 1e3) / peak_exp, 4)})
@@ -963,9 +966,10 @@ def main():
     bound2["note"] = ("the softmax needs the row normalisers before the column sums, so the window product and its "
                       "exponentials run twice; t_exp at the maximum SM clock")
 
-    # ---- the same pass with the caller's log-sum-exp (what a prefill attention kernel keeps per window row): the
-    # statistics sweep and the merge drop out, the entropy call runs the Gram stage on its own.  The normalisers are
-    # prepared once, outside the timed region, by a plain matrix product and logsumexp on the device.
+    # ---- the same pass with the caller's log-sum-exp (what a prefill attention kernel keeps per window row),
+    # through uncomp_compress: the statistics sweep and the merge drop out and the Gram stage rides along with the
+    # column sums, one sweep over K in all.  The normalisers are prepared once, outside the timed region, by a plain
+    # matrix product and logsumexp on the device.
     with_lse = None
     if wl.dtype == "bf16" and not args.no_lse:
         lse = prefill_lse(wl, K, Qw)

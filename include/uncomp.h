@@ -414,6 +414,25 @@ int uncomp_entropy_wide(uncomp_ctx *ctx, const void *d_X, int32_t count, int64_t
 int uncomp_measure_l2_sweep(float *d_A, int32_t rows, int32_t cols, int32_t passes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------------
+ * uncomp_compress -- the whole pass in one call: Section 3.1 - 3.2 (entropy), Section 3.3.3 (budgets, window
+ * scores, selection, per-head cache), in the order that needs the fewest sweeps over K.  Results are those of
+ * uncomp_entropy, uncomp_assign_budgets, uncomp_score_select and uncomp_compact called one after the other
+ * with the same arguments; what changes is the schedule:
+ *   - d_lse given (bf16 keys): ONE sweep over K produces the window scores and the Gram partials of the entropy
+ *     stage together; eigenvalues and budgets follow, then selection and gather.  The staged calls need two
+ *     sweeps for the same result (uncomp_entropy cannot know the normalisers).  The Gram partials are then
+ *     summed per scorer chunk, so entropies can differ from the staged calls in the last bits.
+ *   - d_lse NULL: the staged calls with the Gram + statistics fusion of uncomp_entropy and reuse_stats = 1.
+ * sparams->reuse_stats is ignored.  Arguments, ownership and errors as for the four calls; d_erank is required
+ * here (the budget rule reads it), d_scores may be NULL (scores stay in the workspace), d_layer_group /
+ * d_layer_ctx both NULL or both given. */
+int uncomp_compress(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_strides sK, uncomp_strides sV,
+                    const void *d_Qw, const float *d_lse, const uncomp_entropy_params *eparams,
+                    const uncomp_budget_params *bparams, const uncomp_score_params *sparams, float *d_entropy,
+                    float *d_erank, int32_t *d_budgets, int64_t *d_offsets, int32_t *d_layer_group, int32_t *d_layer_ctx,
+                    float *d_scores, int32_t *d_indices, void *d_Kc, void *d_Vc, void *stream);
+
+/* ---------------------------------------------------------------------------------------------------
  * uncomp_eviction_plan -- Section 3.3.2 "Hidden State Eviction"; Algorithm 2, "compress hidden states":
  * where the prefill cuts the hidden states, read off the layer partition of ONE sequence as
  * uncomp_assign_budgets writes it.  Host function on HOST arrays (copy the L entries of the sequence back

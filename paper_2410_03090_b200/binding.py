@@ -74,6 +74,10 @@ def _load() -> C.CDLL:
     lib.uncomp_score_select.restype = C.c_int
     lib.uncomp_score_select.argtypes = [vp, vp, vp, uncomp_strides, fp, i32p, i64p, C.POINTER(uncomp_score_params),
                                         fp, i32p, vp]
+    lib.uncomp_compress.restype = C.c_int
+    lib.uncomp_compress.argtypes = [vp, vp, vp, uncomp_strides, uncomp_strides, vp, fp, C.POINTER(uncomp_entropy_params),
+                                    C.POINTER(uncomp_budget_params), C.POINTER(uncomp_score_params), fp, fp, i32p, i64p,
+                                    i32p, i32p, fp, i32p, vp, vp, vp]
     lib.uncomp_compact.restype = C.c_int
     lib.uncomp_compact.argtypes = [vp, vp, vp, uncomp_strides, uncomp_strides, i32p, i64p, vp, vp, vp]
     lib.uncomp_set_option.restype = C.c_int
@@ -248,6 +252,25 @@ def uncomp_score_select(ctx: Context, Qw: torch.Tensor, K: torch.Tensor, budgets
                                    _ptr(offsets), C.byref(p), _ptr(scores), _ptr(indices), _stream(stream)),
            "uncomp_score_select")
     return indices
+
+
+def uncomp_compress(ctx: Context, K: torch.Tensor, V: torch.Tensor, Qw: torch.Tensor, entropy_params, budget_params,
+                    score_params, entropy: torch.Tensor, erank: torch.Tensor, budgets: torch.Tensor,
+                    offsets: torch.Tensor, layer_group: Optional[torch.Tensor], layer_ctx: Optional[torch.Tensor],
+                    scores: Optional[torch.Tensor], indices: torch.Tensor, Kc: torch.Tensor, Vc: torch.Tensor,
+                    lse: Optional[torch.Tensor] = None, stream=None) -> None:
+    """The whole pass in one call (every output pre-allocated by the caller).  entropy_params = (k_trunc, center,
+    norm, max_iters), budget_params = (avg_budget, M, n_max, scope, eps, dn, n_last), score_params = (pool_kernel,
+    pool_mode, scale).  With `lse` [B, L, Hq, w] float32 the keys are swept once."""
+    if lse is not None and (lse.dtype != torch.float32 or not lse.is_contiguous()):
+        raise ValueError("lse must be a contiguous float32 tensor [B, L, Hq, w]")
+    ep = uncomp_entropy_params(*entropy_params)
+    bp = uncomp_budget_params(*budget_params)
+    sp = uncomp_score_params(score_params[0], score_params[1], score_params[2], 0)
+    _check(lib.uncomp_compress(ctx.handle, _ptr(K), _ptr(V), strides_of(K), strides_of(V), _ptr(Qw), _ptr(lse),
+                               C.byref(ep), C.byref(bp), C.byref(sp), _ptr(entropy), _ptr(erank), _ptr(budgets),
+                               _ptr(offsets), _ptr(layer_group), _ptr(layer_ctx), _ptr(scores), _ptr(indices), _ptr(Kc),
+                               _ptr(Vc), _stream(stream)), "uncomp_compress")
 
 
 def uncomp_measure_l2_sweep(A: torch.Tensor, passes: int = 1, stream=None) -> None:

@@ -75,6 +75,18 @@ class CompressionPass:
         self.score(K, Qw, stream, eps, dn, n_last, scope, lse)
         return self.compact(K, V, stream)
 
+    def run_one_call(self, K: torch.Tensor, V: torch.Tensor, Qw: torch.Tensor,
+                     stream: Optional[torch.cuda.Stream] = None, eps: float = 0.0, dn: int = 0, n_last: int = 0,
+                     scope: int = 0, lse: Optional[torch.Tensor] = None) -> PassOutput:
+        """The same pass through `uncomp_compress`.  With `lse` the library sweeps the keys once: window scores and
+        the Gram stage of the entropy come out of one kernel."""
+        wl, o = self.wl, self.out
+        ub.uncomp_compress(self.ctx, K, V, Qw, (wl.k_trunc, 1, 0, 0),
+                           (wl.avg_budget, wl.M, wl.n_max, scope, eps, dn, n_last), (wl.pool_kernel, wl.pool_mode, 0.0),
+                           o.entropy, o.erank, o.budgets, o.offsets, o.layer_group, o.layer_ctx, o.scores, o.indices,
+                           o.Kc, o.Vc, lse=lse, stream=stream)
+        return o
+
     def status(self, stream=None) -> int:
         return ub.uncomp_status(self.ctx, stream)
 

@@ -215,7 +215,8 @@ const char *uncomp_profile_slot_name(int slot) {
                                             "evict_logits", "evict_scores", "evict_gather",
                                             "decode_logits", "decode_accumulate", "decode_commit",
                                             "prepare_vote", "prepare_finish",
-                                            "wide_gram", "wide_assemble", "wide_tridiag", "wide_eigen_entropy"};
+                                            "wide_gram", "wide_assemble", "wide_tridiag", "wide_eigen_entropy",
+                                            "gram_score_colsum"};
     return slot >= 0 && slot < kSlotCount ? names[slot] : "";
 }
 
@@ -395,6 +396,77 @@ int uncomp_compact(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_str
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     return UNCOMP_OK;
+}
+
+int uncomp_compress(uncomp_ctx *ctx, const void *d_K, const void *d_V, uncomp_strides sK, uncomp_strides sV,
+                    const void *d_Qw, const float *d_lse, const uncomp_entropy_params *eparams,
+                    const uncomp_budget_params *bparams, const uncomp_score_params *sparams, float *d_entropy,
+                    float *d_erank, int32_t *d_budgets, int64_t *d_offsets, int32_t *d_layer_group, int32_t *d_layer_ctx,
+                    float *d_scores, int32_t *d_indices, void *d_Kc, void *d_Vc, void *stream) {
+    if (!ctx || !eparams || !bparams || !sparams || !d_erank) return UNCOMP_E_NULL;
+    const Plan &p = ctx->plan;
+    const bool tensor_path = p.shape.dtype == UNCOMP_BF16 && !ctx->force_simt;
+    int rc;
+    if (d_lse && tensor_path) {
+        // One sweep over K: the window scores (the caller brings the row normalisers) and the Gram partials of the
+        // entropy stage come out of the same kernel; then eigenvalues, budgets, selection, gather.
+        if (!d_K || !d_Qw || !d_entropy || !d_budgets || !d_offsets || !d_indices) return UNCOMP_E_NULL;
+        if (!aligned16(d_K) || !aligned16(d_Qw) || (reinterpret_cast<uintptr_t>(d_lse) & 3u)) return UNCOMP_E_ALIGN;
+        rc = check_strides(p.shape, sK);
+        if (rc != UNCOMP_OK) return rc;
+        if (eparams->k_trunc < 1 || eparams->max_iters < 0 || (eparams->center != 0 && eparams->center != 1) ||
+            (eparams->norm != 0 && eparams->norm != 1))
+            return UNCOMP_E_PARAM;
+        if (sparams->pool_kernel < 1 || sparams->pool_kernel > 63 || (sparams->pool_kernel & 1) == 0 ||
+            (sparams->pool_mode != 0 && sparams->pool_mode != 1) || !(sparams->scale >= 0.f) || isinf(sparams->scale))
+            return UNCOMP_E_PARAM;
+        if (bparams->scope != 0 && bparams->scope != 1) return UNCOMP_E_PARAM;
+        rc = check_budget_params(p.shape, *bparams);
+        if (rc != UNCOMP_OK) return rc;
+        if ((d_layer_group == nullptr) != (d_layer_ctx == nullptr)) return UNCOMP_E_NULL;
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        uint32_t *d_status = reinterpret_cast<uint32_t *>(ctx->ws + p.off_status);
+        float *partials = reinterpret_cast<float *>(ctx->ws + p.off_gram);
+        float *raw = reinterpret_cast<float *>(ctx->ws + p.off_raw);
+        float *pooled = d_scores ? d_scores : reinterpret_cast<float *>(ctx->ws + p.off_pooled);
+        const UnitAddr addr = make_addr(p.shape, sK);
+        ctx->stats_valid = 0;
+        cudaError_t e = launch_scores_tc(p, d_Qw, d_K, addr, effective_scale(sparams->scale, p.shape.d), d_lse,
+                                         reinterpret_cast<float *>(ctx->ws + p.off_stats_part),
+                                         reinterpret_cast<float *>(ctx->ws + p.off_stats), raw, partials, kScorePhaseColsum,
+                                         d_status, &ctx->tmaps, ctx->prof, st);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        {
+            ProfScope ps(ctx->prof, kSlotEigen, st);
+            e = launch_eigen_f32(p, partials, p.score_splits, *eparams, d_entropy, d_erank, nullptr, d_status, st);
+        }
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        {
+            ProfScope ps(ctx->prof, kSlotBudgets, st);
+            e = launch_budgets(p, d_erank, *bparams, d_budgets, d_offsets, d_layer_group, d_layer_ctx,
+                               reinterpret_cast<int32_t *>(ctx->ws + p.off_rank),
+                               reinterpret_cast<int64_t *>(ctx->ws + p.off_rem), st);
+        }
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        {
+            ProfScope ps(ctx->prof, kSlotPoolSelect, st);
+            e = launch_pool_select(p, raw, pooled, sparams->pool_kernel, sparams->pool_mode, d_budgets, d_offsets,
+                                   d_indices, d_status, st);
+        }
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    } else {
+        // the four calls back to back; bf16 keys without normalisers take the fused Gram + statistics sweep
+        const bool fuse = tensor_path && !d_lse;
+        rc = uncomp_entropy(ctx, d_K, sK, eparams, fuse ? d_Qw : nullptr, sparams->scale, d_entropy, d_erank, nullptr, stream);
+        if (rc != UNCOMP_OK) return rc;
+        rc = uncomp_assign_budgets(ctx, d_erank, bparams, d_budgets, d_offsets, d_layer_group, d_layer_ctx, stream);
+        if (rc != UNCOMP_OK) return rc;
+        uncomp_score_params sp = *sparams;
+        sp.reuse_stats = fuse ? 1 : 0;
+        rc = uncomp_score_select(ctx, d_Qw, d_K, sK, d_lse, d_budgets, d_offsets, &sp, d_scores, d_indices, stream);
+        if (rc != UNCOMP_OK) return rc;
+    }
+    return uncomp_compact(ctx, d_K, d_V, sK, sV, d_indices, d_offsets, d_Kc, d_Vc, stream);
 }
 
 int uncomp_decode_seed(uncomp_ctx *ctx, const float *d_scores, const int32_t *d_indices, const int64_t *d_offsets,

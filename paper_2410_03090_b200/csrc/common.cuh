@@ -82,7 +82,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 enum Slot { kSlotGram = 0, kSlotEigen, kSlotBudgets, kSlotScoreStats, kSlotStatsMerge, kSlotScoreColsum,
             kSlotPoolSelect, kSlotCompact, kSlotGramStats, kSlotEvictLogits, kSlotEvictScores, kSlotEvictGather,
             kSlotDecodeLogits, kSlotDecodeAccumulate, kSlotDecodeCommit, kSlotPrepareVote,
-            kSlotPrepareFinish, kSlotWideGram, kSlotWideAssemble, kSlotWideTridiag, kSlotWideSturm, kSlotCount };
+            kSlotPrepareFinish, kSlotWideGram, kSlotWideAssemble, kSlotWideTridiag, kSlotWideSturm, kSlotGramColsum, kSlotCount };
 enum { kScorePhaseStats = 1, kScorePhaseColsum = 2 };
 struct Profiler;
 void prof_begin(Profiler *p, int slot, cudaStream_t st);
@@ -118,7 +118,8 @@ cudaError_t launch_lse_import(const Plan &p, const float *d_lse, float *d_stats,
                               cudaStream_t st);
 struct TmapCache;
 // phases: kScorePhaseStats (pass A; with d_gram_part != NULL the Gram partials of every (unit, scorer chunk) are
-// produced in the same sweep) and / or kScorePhaseColsum (merge, or the import of d_lse when given, + pass B)
+// produced in the same sweep) and / or kScorePhaseColsum (merge, or the import of d_lse when given, + pass B).
+// kScorePhaseColsum alone with d_gram_part != NULL: pass B and the Gram partials from one sweep (needs d_lse).
 cudaError_t launch_scores_tc(const Plan &p, const void *dQw, const void *dK, const UnitAddr &addr, float scale,
                              const float *d_lse, float *d_stats_part, float *d_stats, float *d_raw, float *d_gram_part,
                              int phases, uint32_t *d_status, TmapCache *cache, Profiler *prof, cudaStream_t st);

@@ -21,6 +21,8 @@
 // Qw K^T is also the MN-major operand of G += K_tile^T K_tile, so the entropy stage costs no second sweep
 // over K.  The Gram block takes the last 128 TMEM columns; the column sums s = K^T 1 are added up by two
 // extra warps (18, 19) with plain global loads of the same tokens (L2 hits), in a fixed order.
+// Mode 3 is pass B with the Gram stage folded in the same way, for callers who bring the row normalisers (their
+// prefill attention kernel's log-sum-exp): entropy stage and scores from ONE sweep over K.
 // Every wait is bounded; a timeout raises UNCOMP_STATUS_TIMEOUT and the CTA drains and exits.
 #include "tc_common.cuh"
 
@@ -39,6 +41,7 @@ constexpr int kMaxStages = 4;
 struct ScoreTail {
     uint64_t full[kMaxStages], empty[kMaxStages], qfull, tfull[2 * kNB], tempty[kNB], gfull;
     uint32_t tmem_base;
+    float sum_xch[kD];     // hand-over of the second column-sum warp (mode 2 and 3)
 };
 
 __host__ __device__ constexpr int score_stages(int MB) { return MB <= 2 ? 4 : (MB == 3 ? 3 : 2); }
@@ -122,13 +125,13 @@ __device__ __forceinline__ float colsum_partial(const uint32_t (&v)[64], float c
 }
 }  // namespace
 
-template <int MB, int MODE>   // MODE 0: pass A, 1: pass B, 2: pass A fused with the Gram stage
+template <int MB, int MODE>   // MODE 0: pass A, 1: pass B, 2: pass A fused with the Gram stage, 3: pass B fused with it
 __global__ void __launch_bounds__(kGramThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant__ CUtensorMap tmapK, int L, int H,
                 int N, int w, int rows, int chunk, int splits, float c_log2, float *__restrict__ stats_part,
                 const float *__restrict__ mprime, float *__restrict__ raw, float *__restrict__ gram_part,
                 const void *__restrict__ Kraw, const UnitAddr kaddr, uint32_t *__restrict__ status) {
-    constexpr bool PASS_B = MODE == 1, GRAM = MODE == 2;
+    constexpr bool PASS_B = MODE == 1 || MODE == 3, GRAM = MODE >= 2;
     // Accumulator buffers (128 TMEM columns each).  An item is one 128-row block of one tile; tile i belongs to
     // softmax group i & 1.  Modes 0 and 1: four buffers, two owned by each group, which it fills alternately
     // with its own items (so each group runs up to two items ahead, independent of the other).  Mode 2: the
@@ -162,7 +165,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = u % H, l = (u / H) % L, b = u / (H * L);
     const int P = N - w;
-    const int limit = PASS_B ? P : N;              // pass B only scores the prefix
+    const int limit = (PASS_B && !GRAM) ? P : N;   // pass B only scores the prefix; the Gram stage needs every token
     const int t0 = c * chunk;
     const int t1 = min(limit, t0 + chunk);
     const int ntiles = t1 > t0 ? (t1 - t0 + kTile - 1) / kTile : 0;
@@ -324,7 +327,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
             for (; r < nrows; ++r) add_bf16x8(acc, ld_stream16(rowp + (int64_t)r * step));
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);   // phases 2 sw, 2 sw + 1
-            float *xch = colsum;                               // unused by the softmax warps in this mode
+            float *xch = T.sum_xch;
             if (sw == 1 && lane < 16) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) xch[ch * 8 + e] = acc[e];
@@ -395,7 +398,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmapQ, const __grid_constant
                 cs[half * 128 + lane_row] = acc;
                 group_barrier(group);
                 const int pos = tile_t0 + lane_row;
-                if (half == 0 && pos < t1 && !dead) raw[(size_t)u * P + pos] = cs[lane_row] + cs[128 + lane_row];
+                if (half == 0 && pos < min(t1, P) && !dead) raw[(size_t)u * P + pos] = cs[lane_row] + cs[128 + lane_row];
             }
         }
         if (!PASS_B) {
@@ -486,6 +489,18 @@ static cudaError_t raise_smem_limit_once() {
 }
 
 template <int MB>
+static cudaError_t raise_smem_limit_mode3() {
+    static bool done[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(score_tc_kernel<MB, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, score_smem(MB));
+    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+    return e;
+}
+
+template <int MB>
 static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, const CUtensorMap &tk, const void *dK,
                                        const UnitAddr &addr, float c_log2,
                                        const float *d_lse, float *d_stats_part, float *d_mprime, float *d_raw,
@@ -508,6 +523,7 @@ static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, con
                                                                       nullptr, nullptr, nullptr, addr, d_status);
     }
     if (phases & kScorePhaseColsum) {
+        const bool with_gram = (phases & kScorePhaseStats) == 0 && d_gram_part != nullptr;   // mode 3
         {
             ProfScope ps(prof, kSlotStatsMerge, st);
             if (d_lse) {
@@ -519,8 +535,17 @@ static cudaError_t launch_scores_tc_mb(const Plan &p, const CUtensorMap &tq, con
                                                                            p.score_splits, d_mprime);
             }
         }
-        ProfScope ps(prof, kSlotScoreColsum, st);
+        ProfScope ps(prof, with_gram ? kSlotGramColsum : kSlotScoreColsum, st);
         const int splitsB = (p.prefix + p.score_chunk - 1) / p.score_chunk;
+        if (with_gram) {
+            e = raise_smem_limit_mode3<MB>();
+            if (e != cudaSuccess) return e;
+            dim3 grid3(p.score_splits, p.units);
+            score_tc_kernel<MB, 3><<<grid3, kGramThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
+                                                                     p.score_splits, c_log2, nullptr, d_mprime, d_raw,
+                                                                     d_gram_part, dK, addr, d_status);
+            return cudaGetLastError();
+        }
         dim3 grid(splitsB, p.units);
         score_tc_kernel<MB, 1><<<grid, kScoreThreads, smem, st>>>(tq, tk, s.L, s.H, s.N, s.w, p.rows, p.score_chunk,
                                                                   splitsB, c_log2, nullptr, d_mprime, d_raw, nullptr,
