@@ -31,13 +31,15 @@ if ROOT not in sys.path:
 # recorded beside them: when the file has changed since the capture, the bench prints null instead.
 NCU_COUNTERS = {
     "source": "paper_2410_03090_b200/csrc/scores_tc.cu",
-    "sha256": "95d4b118eeb6fcb35f3939bddd07669b1930bca35ef0b6c8556135f72cdc081f",
+    "sha256": "5d7704c735797925551e24bea29c1be8724667b424932621e0c8c7a1c44d4428",
     "capture": "ncu --set full, one launch per kernel, c3 scaled to N 16384 x 10 layers; summary in profiles/",
     "kernels": {
-        "gram_score_stats": {"dram_bytes_per_unit_token": (342.071552e6 + 25.281792e6) / (80 * 16384),
-                             "tensor_pipe_pct": 39.7, "xu_pipe_pct": 54.0},
-        "score_colsum": {"dram_bytes_per_unit_token": (340.974080e6 + 7.803136e6) / (80 * 16384),
-                         "tensor_pipe_pct": 35.8, "xu_pipe_pct": 71.5},
+        "gram_score_stats": {"dram_bytes_per_unit_token": (342.482688e6 + 21.898496e6) / (80 * 16384),
+                             "tensor_pipe_pct": 40.0, "xu_pipe_pct": 54.4},
+        "score_colsum": {"dram_bytes_per_unit_token": (340.933120e6 + 7.131136e6) / (80 * 16384),
+                         "tensor_pipe_pct": 33.9, "xu_pipe_pct": 67.9},
+        "gram_score_colsum": {"dram_bytes_per_unit_token": (341.082880e6 + 24.134912e6) / (80 * 16384),
+                              "tensor_pipe_pct": 42.8, "xu_pipe_pct": 57.1},
     },
 }
 EXP_KERNELS = ("score_stats", "score_colsum", "gram_score_stats", "gram_score_colsum")
