@@ -191,12 +191,16 @@ def test_full_size_with_caller_lse(name, n_units):
         assert np.abs(dev_v - v).max() < 1e-3          # the stand-in is a sane normaliser (not a parity claim)
         lse[b, l, h * wl.G:(h + 1) * wl.G] = torch.from_numpy(v.astype(np.float32)).cuda()
     cp = CompressionPass(wl, "cuda")
-    out = cp.run(K, V, Qw, lse=lse)
-    torch.cuda.synchronize()
-    assert cp.status() == 0
-    parity.check_scores(wl, K, Qw, out.scores, units)
-    parity.check_select(wl, out.scores, out.budgets, out.offsets, out.indices, units)
-    parity.check_compact(wl, K, V, out.indices, out.offsets, out.Kc, out.Vc, units[:2])
-    assert int(out.offsets[-1]) == wl.total_rows
+    for one_call in (False, True):          # the staged calls (two sweeps), then uncomp_compress (one sweep: the bench's form)
+        out = cp.run_one_call(K, V, Qw, lse=lse) if one_call else cp.run(K, V, Qw, lse=lse)
+        torch.cuda.synchronize()
+        assert cp.status() == 0
+        parity.check_scores(wl, K, Qw, out.scores, units)
+        parity.check_select(wl, out.scores, out.budgets, out.offsets, out.indices, units)
+        parity.check_compact(wl, K, V, out.indices, out.offsets, out.Kc, out.Vc, units[:2])
+        assert int(out.offsets[-1]) == wl.total_rows
+        if one_call:                         # its entropies come from Gram partials of the fused kernel
+            parity.check_entropy(wl, K, out.entropy, out.erank, units)
+            parity.check_budgets(wl, out.erank, out.budgets, out.offsets, out.layer_group, out.layer_ctx)
     del K, V, Qw, cp, out
     torch.cuda.empty_cache()
