@@ -422,7 +422,12 @@ int uncomp_measure_l2_sweep(float *d_A, int32_t rows, int32_t cols, int32_t pass
  *     stage together; eigenvalues and budgets follow, then selection and gather.  The staged calls need two
  *     sweeps for the same result (uncomp_entropy cannot know the normalisers).  The Gram partials are then
  *     summed per scorer chunk, so entropies can differ from the staged calls in the last bits.
- *   - d_lse NULL: the staged calls with the Gram + statistics fusion of uncomp_entropy and reuse_stats = 1.
+ *   - d_lse NULL (bf16 keys): the Gram + statistics sweep of uncomp_entropy, then eigenvalues and budgets on a
+ *     second stream beside the merge and the column sums (only the selection needs both), joined again before
+ *     the selection.  The second stream is a host object the context creates in the first such call; all work
+ *     is ordered after what `stream` held at the call and `stream` waits for it: same results as the staged
+ *     calls, bit for bit.
+ *   - fp32 keys: the four staged calls.
  * sparams->reuse_stats is ignored.  Arguments, ownership and errors as for the four calls; d_erank is required
  * here (the budget rule reads it), d_scores may be NULL (scores stay in the workspace), d_layer_group /
  * d_layer_ctx both NULL or both given. */
